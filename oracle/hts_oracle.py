@@ -1,0 +1,192 @@
+"""ctypes front end of the plain-C oracle (``hts_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle states, in slow fp64 loops, what the actor
+step and the advantage scan of HTS-RL (arXiv 2012.09849) compute.  It shares
+nothing with the CUDA library; only tests, the smoke check and the CPU-baseline
+leg of the benchmark call it.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hts_oracle.c")
+_LIB = os.path.join(_HERE, "libhts_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over environments)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+class _Weights(C.Structure):
+    _fields_ = [(name, C.c_void_p) for name in (
+        "conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
+        "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.hts_oracle_uniform23.restype = C.c_double
+        _lib.hts_oracle_uniform23.argtypes = [C.c_uint32]
+        _lib.hts_oracle_sample.restype = C.c_int32
+        _lib.hts_oracle_conv_out.restype = C.c_int
+        _lib.hts_oracle_flat_features.restype = C.c_int
+        _lib.hts_oracle_num_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f64(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def num_threads() -> int:
+    return int(lib().hts_oracle_num_threads())
+
+
+def conv_out(extent: int, k: int, s: int) -> int:
+    return int(lib().hts_oracle_conv_out(extent, k, s))
+
+
+def conv2d(x, w, b, stride: int, relu: bool):
+    """x [C,H,W], w [O,C,k,k], b [O] -> y [O,Ho,Wo]; cross-correlation, no padding."""
+    x, w, b = _f64(x), _f64(w), _f64(b)
+    Cc, H, W = x.shape
+    O, C2, k, k2 = w.shape
+    assert C2 == Cc and k == k2 and b.shape == (O,)
+    Ho, Wo = conv_out(H, k, stride), conv_out(W, k, stride)
+    y = np.empty((O, Ho, Wo), dtype=np.float64)
+    lib().hts_oracle_conv2d(_p(x), Cc, H, W, _p(w), _p(b), O, k, stride, int(relu), _p(y))
+    return y
+
+
+def linear(x, w, b, relu: bool):
+    x, w, b = _f64(x), _f64(w), _f64(b)
+    O, I = w.shape
+    y = np.empty(O, dtype=np.float64)
+    lib().hts_oracle_linear(_p(x), I, _p(w), _p(b), O, int(relu), _p(y))
+    return y
+
+
+class Weights:
+    """fp64 copies of the twelve parameter tensors (PyTorch OIHW / [out,in] layout)."""
+    NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
+             "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
+
+    def __init__(self, params: dict):
+        self.arr = {k: _f64(params[k]) for k in self.NAMES}
+        self.A = self.arr["pi_w"].shape[0]
+        self.C = self.arr["conv1_w"].shape[1]
+        self.c = _Weights(**{k: _p(v) for k, v in self.arr.items()})
+
+
+def policy_forward(wt: Weights, obs: np.ndarray, taps: bool = False):
+    """obs u8 [n,C,H,W] -> dict(logits [n,A], value [n], optional layer taps)."""
+    obs = np.ascontiguousarray(obs, dtype=np.uint8)
+    n, Cc, H, W = obs.shape
+    assert Cc == wt.C
+    A = wt.A
+    h1, w1 = conv_out(H, 8, 4), conv_out(W, 8, 4)
+    h2, w2 = conv_out(h1, 4, 2), conv_out(w1, 4, 2)
+    h3, w3 = conv_out(h2, 3, 1), conv_out(w2, 3, 1)
+    assert wt.arr["fc_w"].shape == (512, 64 * h3 * w3)
+    out = {"logits": np.empty((n, A)), "value": np.empty(n)}
+    t1 = t2 = t3 = t4 = None
+    if taps:
+        t1 = np.empty((n, 32, h1, w1)); t2 = np.empty((n, 64, h2, w2))
+        t3 = np.empty((n, 64, h3, w3)); t4 = np.empty((n, 512))
+        out.update(conv1=t1, conv2=t2, conv3=t3, fc=t4)
+    lib().hts_oracle_policy_forward(C.byref(wt.c), _p(obs), n, Cc, H, W, A,
+                                    _p(out["logits"]), _p(out["value"]),
+                                    _p(t1), _p(t2), _p(t3), _p(t4))
+    return out
+
+
+def log_softmax(logits):
+    """logits [A] -> (log pi [A], entropy) in nats (Eq. 3's H)."""
+    logits = _f64(logits)
+    A = logits.shape[0]
+    lp = np.empty(A)
+    ent = C.c_double()
+    lib().hts_oracle_log_softmax(_p(logits), A, _p(lp), C.byref(ent))
+    return lp, ent.value
+
+
+def philox4x32_10(ctr, key):
+    c = (C.c_uint32 * 4)(*[int(v) & 0xFFFFFFFF for v in ctr])
+    k = (C.c_uint32 * 2)(*[int(v) & 0xFFFFFFFF for v in key])
+    o = (C.c_uint32 * 4)()
+    lib().hts_oracle_philox4x32_10(c, k, o)
+    return tuple(int(v) for v in o)
+
+
+def uniform23(word: int) -> float:
+    return float(lib().hts_oracle_uniform23(C.c_uint32(int(word) & 0xFFFFFFFF)))
+
+
+def action_uniforms(seed: int, env_id: int, t: int, A: int):
+    """-> (words u32 [A], uniforms f64 [A]) for (seed, env_id, t)."""
+    words = np.empty(A, dtype=np.uint32)
+    u = np.empty(A, dtype=np.float64)
+    lib().hts_oracle_action_uniforms(C.c_uint64(seed), C.c_int32(env_id), C.c_int32(t), A,
+                                     _p(words), _p(u))
+    return words, u
+
+
+def sample(logits, seed: int, env_id: int, t: int):
+    """-> dict(action, scores [A], gap, runner_up): Gumbel-max on (seed, env_id, t)."""
+    logits = _f64(logits)
+    A = logits.shape[0]
+    scores = np.empty(A)
+    gap = C.c_double()
+    ru = C.c_int32()
+    a = lib().hts_oracle_sample(_p(logits), A, C.c_uint64(seed), C.c_int32(env_id),
+                                C.c_int32(t), _p(scores), C.byref(gap), C.byref(ru))
+    return {"action": int(a), "scores": scores, "gap": gap.value, "runner_up": ru.value}
+
+
+def policy_step(wt: Weights, obs, env_ids, t, seed: int, t_per_env=None):
+    """The whole actor step on a batch. Returns a dict of per-env arrays."""
+    obs = np.ascontiguousarray(obs, dtype=np.uint8)
+    n, Cc, H, W = obs.shape
+    env_ids = np.ascontiguousarray(env_ids, dtype=np.int32)
+    assert env_ids.shape == (n,)
+    tp = None if t_per_env is None else np.ascontiguousarray(t_per_env, dtype=np.int32)
+    A = wt.A
+    out = {"actions": np.empty(n, np.int32), "logp": np.empty(n), "values": np.empty(n),
+           "entropy": np.empty(n), "logits": np.empty((n, A)), "gap": np.empty(n),
+           "runner_up": np.empty(n, np.int32)}
+    lib().hts_oracle_policy_step(C.byref(wt.c), _p(obs), _p(env_ids), _p(tp), C.c_int32(int(t)),
+                                 C.c_uint64(seed), n, Cc, H, W, A,
+                                 _p(out["actions"]), _p(out["logp"]), _p(out["values"]),
+                                 _p(out["entropy"]), _p(out["logits"]), _p(out["gap"]),
+                                 _p(out["runner_up"]))
+    return out
+
+
+def gae(rewards, values, dones, bootstrap, gamma: float, lam: float):
+    """[T,N] fp32 rewards/values, u8 dones, [N] bootstrap -> (adv, ret) fp64 [T,N]."""
+    r = np.ascontiguousarray(rewards, dtype=np.float32)
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    d = np.ascontiguousarray(dones, dtype=np.uint8)
+    b = np.ascontiguousarray(bootstrap, dtype=np.float32)
+    T, N = r.shape
+    assert v.shape == (T, N) and d.shape == (T, N) and b.shape == (N,)
+    adv = np.empty((T, N)); ret = np.empty((T, N))
+    lib().hts_oracle_gae(_p(r), _p(v), _p(d), _p(b), C.c_double(gamma), C.c_double(lam),
+                         T, N, _p(adv), _p(ret))
+    return adv, ret
