@@ -1,0 +1,172 @@
+/*
+ * hts.h -- C ABI of the HTS-RL hot-path library for NVIDIA B200 (sm_100a).
+ *
+ * Two operations of the synchronous actor-critic pipeline of "High-Throughput
+ * Synchronous Deep RL" (arXiv 2012.09849) are exported:
+ *
+ *   hts_policy_step  the batched actor step (Section 4.1, "Asynchronous actors and
+ *                    executors"): one forward pass of the policy-value network of
+ *                    Appendix F.1 / F.2 over all observations handed in, then one
+ *                    sampled action per observation whose randomness depends only
+ *                    on (seed, env_id, t), never on how the batch was grouped.
+ *   hts_gae          the return / advantage computation over the [T,N] rollout
+ *                    storage that feeds the learner (Section 3, "Actor-Critic
+ *                    Algorithms": n-step truncated return; GAE generalises it).
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *   - Plain C: no exceptions or aborts cross this boundary; every call returns an
+ *     hts_status.  Invalid arguments are detected on the host before any launch.
+ *   - "DEVICE" pointers are CUDA device memory of the current device, owned by the
+ *     caller; the library never frees them and does not keep them after the
+ *     stream work of the call.  "HOST" pointers are ordinary host memory.
+ *   - Calls taking a `cuda_stream` (a cudaStream_t passed as void*, NULL = legacy
+ *     default stream) only enqueue work on that stream and do not synchronise.
+ *   - Output buffers must not overlap input buffers or each other.
+ *   - There is no CPU fallback: without a CUDA device calls return HTS_ERR_CUDA.
+ */
+#ifndef HTS_H_
+#define HTS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hts_ctx hts_ctx; /* opaque: packed weights + activation workspace */
+
+typedef enum {
+    HTS_OK = 0,
+    HTS_ERR_INVALID_ARG = 1, /* NULL pointer, overlap, n outside 1..max_batch, bad gamma/lambda ... */
+    HTS_ERR_SHAPE = 2,       /* network geometry not supported                       */
+    HTS_ERR_ALLOC = 3,       /* device or host allocation failed                     */
+    HTS_ERR_CUDA = 4,        /* a CUDA runtime call failed (see hts_last_cuda_error) */
+    HTS_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out                   */
+    HTS_ERR_UNSUPPORTED = 6  /* valid request that this build does not implement     */
+} hts_status;
+
+/* weight_dtype */
+#define HTS_DTYPE_FP32 0 /* fp32 weights, fp32 CUDA-core arithmetic: the check path   */
+#define HTS_DTYPE_BF16 1 /* bf16 weights, tensor-core path with fp32 accumulation     */
+
+/* Network geometry.  The layers are fixed by Appendix F.1 / F.2 of the paper:
+ * conv 32@8x8/4 -> conv 64@4x4/2 -> conv 64@3x3/1 -> FC 512 -> {policy over
+ * num_actions, scalar value}; no padding, ReLU after the four hidden layers, input
+ * scaled by 1/255.  C,H,W describe one uint8 observation (H,W multiples of 4 and
+ * large enough that every layer has at least one output); 1 <= num_actions <= 64. */
+typedef struct {
+    int32_t C, H, W;
+    int32_t num_actions;
+    int32_t weight_dtype; /* HTS_DTYPE_*                                  */
+    int32_t max_batch;    /* largest n any later hts_policy_step may pass */
+} hts_net_desc;
+
+/* The twelve parameter tensors, PyTorch layouts, all DEVICE pointers, element type
+ * given by weight_dtype (float, or bf16 stored as 16-bit patterns).
+ * F = 64*H3*W3 is the flattened conv3 output; FC column f = c*H3*W3 + h*W3 + w.   */
+typedef struct {
+    const void *conv1_w, *conv1_b; /* [32,C,8,8], [32]  */
+    const void *conv2_w, *conv2_b; /* [64,32,4,4], [64] */
+    const void *conv3_w, *conv3_b; /* [64,64,3,3], [64] */
+    const void *fc_w, *fc_b;       /* [512,F], [512]    */
+    const void *pi_w, *pi_b;       /* [A,512], [A]      */
+    const void *v_w, *v_b;         /* [1,512], [1]      */
+} hts_weights;
+
+/* Create a context for one network geometry on the current device.  Allocates the
+ * packed-weight store and an activation workspace sized for max_batch (device
+ * memory, freed by hts_policy_destroy).  Errors: INVALID_ARG, SHAPE, ALLOC, CUDA. */
+hts_status hts_policy_create(const hts_net_desc *desc, hts_ctx **out);
+
+/* Repack the caller's weights into the library's internal layouts on `cuda_stream`.
+ * May be called again at any time (e.g. after each learner update: the parameter
+ * hand-over of Section 4.1 "Delayed gradient"); steps enqueued later on the same
+ * stream see the new weights.  The caller's buffers are read during the stream
+ * work of this call only.                                                        */
+hts_status hts_policy_load_weights(hts_ctx *ctx, const hts_weights *w, void *cuda_stream);
+
+/* The batched actor step (Section 4.1; network of Appendix F.1/F.2; outputs are
+ * the quantities of Eq. 3/4: log pi(a|s), V(s), H(pi(.|s)) in nats).
+ *   obs        DEVICE u8  [n,C,H,W]   raw frames, NCHW
+ *   env_ids    DEVICE i32 [n]         global environment index of each row (>= 0;
+ *                                      duplicates allowed)
+ *   t_per_env  DEVICE i32 [n] or NULL per-row time index; NULL = every row uses `t`
+ *   seed                               64-bit run seed
+ *   n                                  1..max_batch, any value (no tile multiple needed)
+ *   actions    DEVICE i32 [n]   out   Gumbel-max sample: argmax_a logit_a - log(-log u_a),
+ *                                      u_a from Philox4x32-10 with counter
+ *                                      (env_id, t, a/4, 0), key (seed_lo, seed_hi),
+ *                                      word a%4, u = ((word>>9)+0.5)*2^-23; ties -> lowest a
+ *   logp, values, entropy  DEVICE f32 [n]  out
+ *   logits_or_null  DEVICE f32 [n,A] or NULL  out  raw policy logits (parity tap)
+ * Each row's outputs are independent of n, of the row's position and of the other
+ * rows.  Errors: INVALID_ARG (NULL, n out of range, overlap), CUDA, UNSUPPORTED
+ * (weights not loaded).                                                           */
+hts_status hts_policy_step(hts_ctx *ctx, const uint8_t *obs, const int32_t *env_ids,
+                           const int32_t *t_per_env, int32_t t, uint64_t seed, int32_t n,
+                           int32_t *actions, float *logp, float *values, float *entropy,
+                           float *logits_or_null, void *cuda_stream);
+
+/* Same operation with HOST buffers: copies obs/env_ids/t_per_env to the device,
+ * runs the step, copies the four outputs (and logits if asked) back and waits for
+ * them.  Uses staging buffers owned by the context (allocated at create time).
+ * Pinned host memory makes the copies asynchronous but is not required.           */
+hts_status hts_policy_step_host(hts_ctx *ctx, const uint8_t *obs, const int32_t *env_ids,
+                                const int32_t *t_per_env, int32_t t, uint64_t seed, int32_t n,
+                                int32_t *actions, float *logp, float *values, float *entropy,
+                                float *logits_or_null, void *cuda_stream);
+
+/* Parity tap: convert the hidden activation left in the workspace by the most
+ * recent hts_policy_step on this context into fp32 NCHW.
+ *   layer 1..3 -> conv outputs [n,32,H1,W1], [n,64,H2,W2], [n,64,H3,W3]; 4 -> FC [n,512]
+ *   out  DEVICE f32, n = rows of that step.  Enqueued on cuda_stream.             */
+hts_status hts_policy_read_activation(hts_ctx *ctx, int32_t layer, int32_t n, float *out,
+                                      void *cuda_stream);
+
+/* Parity tap for the sampler's random stream (Section 4.1: the per-observation
+ * pseudo-random number): writes the num_actions uniforms that hts_policy_step
+ * uses for each row, computed by the same device function.
+ *   env_ids DEVICE i32 [n]; t_per_env DEVICE i32 [n] or NULL; out DEVICE f32 [n,num_actions] */
+hts_status hts_action_uniforms(const int32_t *env_ids, const int32_t *t_per_env, int32_t t,
+                               uint64_t seed, int32_t n, int32_t num_actions, float *out,
+                               void *cuda_stream);
+
+/* Reads and clears the device status word of the context (set by a bounded wait
+ * that ran out).  Synchronises with the device.  HTS_OK if nothing was recorded.  */
+hts_status hts_last_async_error(hts_ctx *ctx);
+
+void hts_policy_destroy(hts_ctx *ctx);
+
+/* Advantages and returns over the rollout storage (Section 3: with lambda = 1,
+ * returns[t] is the n-step truncated return with n = T - t):
+ *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t          V_T = bootstrap
+ *   A_t     = delta_t + gamma lambda (1-d_t) A_{t+1}     A_T = 0
+ *   R_t     = A_t + V_t
+ *   rewards, values  DEVICE f32 [T,N] time-major;  dones DEVICE u8 [T,N], non-zero =
+ *   the transition taken at step t ended the episode;  bootstrap DEVICE f32 [N];
+ *   advantages, returns  DEVICE f32 [T,N] out.   0 <= gamma, lambda <= 1, finite.
+ * T >= 1, N >= 1.  Errors: INVALID_ARG, CUDA.                                      */
+hts_status hts_gae(const float *rewards, const float *values, const uint8_t *dones,
+                   const float *bootstrap, float gamma, float lambda, int32_t T, int32_t N,
+                   float *advantages, float *returns, void *cuda_stream);
+
+/* Same with HOST buffers; copies in, computes, copies out and waits.  Staging
+ * memory is a library-owned device buffer that grows on demand (not thread safe). */
+hts_status hts_gae_host(const float *rewards, const float *values, const uint8_t *dones,
+                        const float *bootstrap, float gamma, float lambda, int32_t T,
+                        int32_t N, float *advantages, float *returns, void *cuda_stream);
+
+/* Number of kernel launches this library has enqueued since it was loaded
+ * (all contexts, all streams); for launch accounting by a benchmark.              */
+uint64_t hts_launch_count(void);
+
+/* Text of the last CUDA runtime error seen by this library on the calling thread
+ * (empty string if none).                                                         */
+const char *hts_last_cuda_error(void);
+
+const char *hts_status_string(hts_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HTS_H_ */

@@ -1,0 +1,62 @@
+// Shared declarations of the library's translation units (host side + small device helpers).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "hts.h"
+
+namespace hts {
+
+// ---- launch accounting and error capture --------------------------------------------------
+void note_launch(int count = 1);
+hts_status cuda_fail(cudaError_t e, const char* where);   // records text, returns HTS_ERR_CUDA
+#define HTS_CUDA(call)                                                        \
+    do {                                                                      \
+        cudaError_t e__ = (call);                                             \
+        if (e__ != cudaSuccess) return ::hts::cuda_fail(e__, #call);          \
+    } while (0)
+#define HTS_LAUNCH_CHECK(name)                                                \
+    do {                                                                      \
+        ::hts::note_launch();                                                 \
+        cudaError_t e__ = cudaGetLastError();                                 \
+        if (e__ != cudaSuccess) return ::hts::cuda_fail(e__, name);           \
+    } while (0)
+
+inline int conv_out(int extent, int k, int s) { return (extent - k) / s + 1; }
+
+// Geometry of the fixed four-layer network for one observation shape.
+struct Geometry {
+    int C, H, W, A;
+    int H1, W1, H2, W2, H3, W3, F;
+};
+
+// ---- the fp32 CUDA-core path (check path; also the fallback arithmetic for bf16 weights) ---
+struct RefWeights {            // fp32 device copies in PyTorch layouts
+    float *w1, *b1, *w2, *b2, *w3, *b3, *wfc, *bfc;
+    float *whead, *bhead;      // [A+1,512], [A+1]: policy rows then the value row
+};
+struct RefWorkspace { float *a1, *a2, *a3, *h; };   // NCHW fp32 activations, [n,512]
+
+hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& src,
+                               const RefWeights& dst, cudaStream_t s);
+hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
+                       const uint8_t* obs, int n, cudaStream_t s);
+
+// ---- heads + distribution + sampling epilogue (both paths) --------------------------------
+// h_partials: [num_splits][n][512] fp32.  If fc_bias != nullptr the hidden vector is
+// relu(fc_bias + sum over splits in index order), else it is h_partials[0] as is.
+hts_status launch_heads(const float* h_partials, int num_splits, size_t split_stride,
+                        const float* fc_bias, const float* whead, const float* bhead, int A,
+                        const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
+                        uint64_t seed, int n, int32_t* actions, float* logp, float* values,
+                        float* entropy, float* logits, float* h_out, cudaStream_t s);
+
+hts_status launch_uniforms(const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed, int n,
+                           int A, float* out, cudaStream_t s);
+
+// ---- advantage scan -------------------------------------------------------------------------
+hts_status launch_gae(const float* rewards, const float* values, const uint8_t* dones,
+                      const float* bootstrap, float gamma, float lambda, int T, int N,
+                      float* adv, float* ret, cudaStream_t s);
+
+}  // namespace hts

@@ -1,0 +1,160 @@
+// Policy / value heads and the sampling epilogue of the actor step.
+//
+// One warp per observation.  The warp forms the 512 hidden units (summing the FC split-K
+// partials in index order when asked), takes the A+1 head dot products, then the policy
+// distribution (log-softmax, entropy in nats: the H(pi(.|s)) of Eq. 3) and one action by
+// Gumbel-max.  The uniforms come from Philox4x32-10 (Salmon et al., SC'11) with counter
+// (env_id, t, a/4, 0) and key (seed_lo, seed_hi): the per-observation pseudo-random number
+// of Section 4.1, so the action is a function of (seed, env_id, t) and the logits alone.
+#include "common.cuh"
+
+namespace hts {
+namespace {
+
+constexpr int kHidden = 512;
+constexpr int kMaxActions = 64;
+
+__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1)
+{
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+    const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+}
+
+__device__ __forceinline__ uint32_t philox_word(uint32_t env, uint32_t t, uint32_t block, uint32_t lane4,
+                                                uint32_t k0, uint32_t k1)
+{
+    uint32_t c[4] = {env, t, block, 0u};
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        philox_round(c, k0, k1);
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return lane4 == 0 ? c[0] : lane4 == 1 ? c[1] : lane4 == 2 ? c[2] : c[3];
+}
+
+// u = ((word >> 9) + 1/2) * 2^-23: 23 bits so that the value is exact in fp32 and inside (0,1)
+__device__ __forceinline__ float action_uniform(uint32_t env, uint32_t t, int a, uint32_t k0, uint32_t k1)
+{
+    const uint32_t word = philox_word(env, t, (uint32_t)a >> 2, (uint32_t)a & 3u, k0, k1);
+    return ((float)(word >> 9) + 0.5f) * (1.0f / 8388608.0f);
+}
+
+__global__ void uniforms_kernel(const int32_t* __restrict__ env_ids, const int32_t* __restrict__ t_per_env,
+                                int32_t t_scalar, uint32_t k0, uint32_t k1, int n, int A, float* __restrict__ out)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)n * A) return;
+    const int e = (int)(i / A), a = (int)(i % A);
+    out[i] = action_uniform((uint32_t)env_ids[e], (uint32_t)(t_per_env ? t_per_env[e] : t_scalar), a, k0, k1);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    return v;
+}
+
+__global__ void __launch_bounds__(256)
+heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_stride,
+             const float* __restrict__ fc_bias, const float* __restrict__ whead,
+             const float* __restrict__ bhead, int A, const int32_t* __restrict__ env_ids,
+             const int32_t* __restrict__ t_per_env, int32_t t_scalar, uint32_t key0, uint32_t key1,
+             int n, int32_t* __restrict__ actions, float* __restrict__ logp,
+             float* __restrict__ values, float* __restrict__ entropy, float* __restrict__ logits_out,
+             float* __restrict__ h_out)
+{
+    __shared__ float s_out[8][kMaxActions + 1];
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int e = blockIdx.x * 8 + wib;
+    if (e >= n) return;
+
+    float h[kHidden / 32];
+#pragma unroll
+    for (int i = 0; i < kHidden / 32; ++i) {
+        const int f = lane + 32 * i;
+        float v = h_partials[(size_t)e * kHidden + f];
+        if (fc_bias) {
+            for (int sp = 1; sp < num_splits; ++sp) v += h_partials[sp * split_stride + (size_t)e * kHidden + f];
+            v += fc_bias[f];
+            v = v > 0.f ? v : 0.f;
+        }
+        h[i] = v;
+        if (h_out) h_out[(size_t)e * kHidden + f] = v;
+    }
+    for (int o = 0; o <= A; ++o) {
+        const float* wr = whead + (size_t)o * kHidden;
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < kHidden / 32; ++i) acc = fmaf(wr[lane + 32 * i], h[i], acc);
+        acc = warp_sum(acc);
+        if (lane == 0) s_out[wib][o] = acc + bhead[o];
+    }
+    __syncwarp();
+    const float* lg = s_out[wib];
+
+    float m = -INFINITY;
+    for (int a = lane; a < A; a += 32) m = fmaxf(m, lg[a]);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+    float z = 0.f;
+    for (int a = lane; a < A; a += 32) z += expf(lg[a] - m);
+    z = warp_sum(z);
+    const float lse = m + logf(z);
+    float ent = 0.f;
+    for (int a = lane; a < A; a += 32) { const float lp = lg[a] - lse; ent -= expf(lp) * lp; }
+    ent = warp_sum(ent);
+
+    const uint32_t env = (uint32_t)env_ids[e];
+    const uint32_t tt = (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
+    float best = -INFINITY; int best_a = 0x7fffffff;
+    for (int a = lane; a < A; a += 32) {
+        const float u = action_uniform(env, tt, a, key0, key1);
+        const float score = lg[a] - logf(-logf(u));
+        if (score > best) { best = score; best_a = a; }                        // ascending a: ties keep the lowest
+    }
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, k);
+        const int oa = __shfl_xor_sync(0xffffffffu, best_a, k);
+        if (ob > best || (ob == best && oa < best_a)) { best = ob; best_a = oa; }
+    }
+    if (logits_out) for (int a = lane; a < A; a += 32) logits_out[(size_t)e * A + a] = lg[a];
+    if (lane == 0) {
+        actions[e] = best_a;
+        logp[e] = lg[best_a] - lse;
+        values[e] = lg[A];
+        entropy[e] = ent;
+    }
+}
+
+}  // namespace
+
+hts_status launch_heads(const float* h_partials, int num_splits, size_t split_stride,
+                        const float* fc_bias, const float* whead, const float* bhead, int A,
+                        const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
+                        uint64_t seed, int n, int32_t* actions, float* logp, float* values,
+                        float* entropy, float* logits, float* h_out, cudaStream_t s)
+{
+    heads_kernel<<<(n + 7) / 8, 256, 0, s>>>(h_partials, num_splits, split_stride, fc_bias, whead, bhead, A,
+                                           env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu),
+                                           (uint32_t)(seed >> 32), n, actions, logp, values, entropy,
+                                           logits, h_out);
+    HTS_LAUNCH_CHECK("heads_kernel");
+    return HTS_OK;
+}
+
+hts_status launch_uniforms(const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed, int n,
+                           int A, float* out, cudaStream_t s)
+{
+    const size_t total = (size_t)n * A;
+    uniforms_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(env_ids, t_per_env, t,
+                                                                  (uint32_t)(seed & 0xffffffffu),
+                                                                  (uint32_t)(seed >> 32), n, A, out);
+    HTS_LAUNCH_CHECK("uniforms_kernel");
+    return HTS_OK;
+}
+
+}  // namespace hts
