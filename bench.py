@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the HTS-RL hot path on B200: actor env-steps/s over whole rollouts.
+
+One step = one rollout of the "ppo_atari_large" workload: T=128 batched actor steps over
+N=1024 environments (uint8 4x84x84 observations from a ring of pre-generated batches larger
+than L2) writing values/log-probs/actions into one of two rollout storages, plus the GAE scan
+of the previous rollout on a second stream (its bootstrap is the value row 0 of the rollout
+being collected), as in the paper's concurrent rollout and learning.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  With N > 1 (torchrun) every rank runs the same workload on
+its own range of environment ids; there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import hts_workloads as wl  # noqa: E402
+
+WORKLOAD = 3                       # hts_workloads.CONFIGS index
+METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
+UNIT = "env-steps/s"
+SEED = 0x5EED
+
+
+def macs_per_env_step(cfg) -> int:
+    h1, w1 = wl.conv_out(cfg.H, 8, 4), wl.conv_out(cfg.W, 8, 4)
+    h2, w2 = wl.conv_out(h1, 4, 2), wl.conv_out(w1, 4, 2)
+    h3, w3 = wl.conv_out(h2, 3, 1), wl.conv_out(w2, 3, 1)
+    return (32 * h1 * w1 * cfg.C * 64 + 64 * h2 * w2 * 32 * 16 + 64 * h3 * w3 * 64 * 9
+            + 512 * 64 * h3 * w3 + (cfg.A + 1) * 512)
+
+
+def layer_macs(cfg) -> dict:
+    h1, w1 = wl.conv_out(cfg.H, 8, 4), wl.conv_out(cfg.W, 8, 4)
+    h2, w2 = wl.conv_out(h1, 4, 2), wl.conv_out(w1, 4, 2)
+    h3, w3 = wl.conv_out(h2, 3, 1), wl.conv_out(w2, 3, 1)
+    return {"conv1": 32 * h1 * w1 * cfg.C * 64, "conv2": 64 * h2 * w2 * 32 * 16,
+            "conv3": 64 * h3 * w3 * 64 * 9, "fc": 512 * 64 * h3 * w3, "heads": (cfg.A + 1) * 512}
+
+
+def measured_peaks() -> tuple[dict, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = sorted(sm)[len(sm) // 2:] if sm else []           # upper half: samples under load
+        return {"sm_mhz": float(np.median(busy)) if busy else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args) -> None:
+    """The CPU oracle as it stands, on a bounded sample per step, on this host's cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import hts_oracle as orc
+    cfg = wl.CONFIGS[WORKLOAD]
+    wt = orc.Weights(wl.make_weights(cfg))
+    r, v, d, b = wl.make_rollout(cfg)
+    sample_rows = 512
+    env_ids = np.arange(sample_rows, dtype=np.int32)
+    obs = [wl.make_obs(cfg, sample_rows, batch_index=i) for i in range(2)]
+
+    def one(i):
+        t0 = time.perf_counter()
+        orc.policy_step(wt, obs[i % 2], env_ids, i, SEED)
+        t1 = time.perf_counter()
+        orc.gae(r, v, d, b, cfg.gamma, cfg.lam)
+        t2 = time.perf_counter()
+        return t1 - t0, t2 - t1
+
+    for i in range(args.warmup):
+        one(i)
+    ta = tg = 0.0
+    for i in range(args.steps):
+        a, g = one(i)
+        ta += a; tg += g
+    per_env_step = ta / (args.steps * sample_rows) + tg / (args.steps * cfg.T * cfg.N)
+    value = 1.0 / per_env_step
+    sample = (f"per step: one actor step on {sample_rows} of {cfg.N} envs + one full GAE [{cfg.T},{cfg.N}]; "
+              f"rate = 1/(actor s per env-step + GAE s per element)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * (ta + tg) / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "N": cfg.N, "T": cfg.T, "obs": [cfg.C, cfg.H, cfg.W], "actions": cfg.A},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args) -> None:
+    import torch
+    import paper_2012_09849_b200 as hts
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = wl.CONFIGS[WORKLOAD]
+    T, N, A = cfg.T, cfg.N, cfg.A
+    obs_bytes = cfg.C * cfg.H * cfg.W
+    peaks, peak_kind = measured_peaks()
+    l2 = torch.cuda.get_device_properties(local).L2_cache_size
+    ring = max(8, -(-2 * l2 // (N * obs_bytes)))                 # ring of distinct batches > 2x L2
+    dev = torch.device("cuda", local)
+
+    ctx = hts.hts_policy_create(cfg.C, cfg.H, cfg.W, A, hts.HTS_DTYPE_BF16, N)
+    params = wl.make_weights(cfg)
+    dev_w = hts.weights_to_device(params, hts.HTS_DTYPE_BF16, dev)
+    hts.hts_policy_load_weights(ctx, dev_w)
+    obs_host = [torch.from_numpy(wl.make_obs(cfg, N, batch_index=i)).pin_memory() for i in range(ring)]
+    obs_dev = [o.to(dev) for o in obs_host]
+    env_ids = torch.arange(rank * N, (rank + 1) * N, dtype=torch.int32, device=dev)
+    r_np, _, d_np, _ = wl.make_rollout(cfg)
+    rewards, dones = torch.from_numpy(r_np).to(dev), torch.from_numpy(d_np).to(dev)
+
+    class Storage:                                               # one of the two rollout storages
+        def __init__(self):
+            self.actions = torch.empty(T, N, dtype=torch.int32, device=dev)
+            self.logp = torch.empty(T, N, dtype=torch.float32, device=dev)
+            self.values = torch.empty(T, N, dtype=torch.float32, device=dev)
+            self.entropy = torch.empty(T, N, dtype=torch.float32, device=dev)
+            self.adv = torch.empty(T, N, dtype=torch.float32, device=dev)
+            self.ret = torch.empty(T, N, dtype=torch.float32, device=dev)
+            self.filled = torch.cuda.Event()                     # all T actor steps written
+            self.row0 = torch.cuda.Event()                       # value row 0 written
+            self.consumed = torch.cuda.Event()                   # GAE has read it
+            # raw row addresses, so the timed loop does no tensor slicing
+            self.p_act = [self.actions[t].data_ptr() for t in range(T)]
+            self.p_logp = [self.logp[t].data_ptr() for t in range(T)]
+            self.p_val = [self.values[t].data_ptr() for t in range(T)]
+            self.p_ent = [self.entropy[t].data_ptr() for t in range(T)]
+    store = [Storage(), Storage()]
+    s_act, s_gae = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    p_obs = [o.data_ptr() for o in obs_dev]
+    p_ids, h_act_stream, h_gae_stream = env_ids.data_ptr(), s_act.cuda_stream, s_gae.cuda_stream
+
+    def rollout(k: int):
+        cur, prev = store[k % 2], store[(k + 1) % 2]
+        s_act.wait_event(cur.consumed)                           # storage free again (role swap)
+        for t in range(T):
+            hts.hts_policy_step(ctx, p_obs[(k * T + t) % ring], p_ids, None, t, SEED + k, N,
+                                cur.p_act[t], cur.p_logp[t], cur.p_val[t], cur.p_ent[t], None, h_act_stream)
+            if t == 0:
+                cur.row0.record(s_act)
+        cur.filled.record(s_act)
+        # GAE of the previous rollout on the second stream; bootstrap = V of this rollout's first states
+        s_gae.wait_event(prev.filled)
+        s_gae.wait_event(cur.row0)
+        hts.hts_gae(rewards, prev.values, dones, cur.p_val[0], cfg.gamma, cfg.lam, T, N, prev.adv, prev.ret,
+                    h_gae_stream)
+        prev.consumed.record(s_gae)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for s in store:
+        s.consumed.record(s_gae); s.filled.record(s_act); s.row0.record(s_act)
+    rollout(-1)                                                  # fills storage 1 so the first GAE has input
+    for k in range(args.warmup):
+        rollout(k)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = hts.hts_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s_act)
+    for k in range(args.steps):
+        rollout(args.warmup + k)
+    s_act.wait_stream(s_gae)
+    e1.record(s_act)
+    barrier()
+    launches = hts.hts_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tms = torch.tensor([ms], device=dev); dist.all_reduce(tms, op=dist.ReduceOp.MAX); ms = float(tms.item())
+    value = world * args.steps * T * N / (ms * 1e-3)
+
+    # ---- per-kernel device times over the same region (second pass, events around each kernel)
+    hts.hts_policy_profile(ctx, True)
+    for k in range(min(args.steps, 4096 // T)):
+        rollout(args.warmup + args.steps + k)
+    torch.cuda.synchronize()
+    hts.hts_policy_profile(ctx, False)
+    kern = {}
+    for i in range(5):
+        tot, cnt = hts.hts_policy_profile_read(ctx, i)
+        kern[hts.hts_policy_kernel_name(i)] = {"ms_total": tot, "launches": cnt,
+                                               "us_per_launch": 1e3 * tot / max(cnt, 1)}
+    # GAE alone, cold (inputs evicted by a write larger than L2 between launches)
+    flush = torch.empty(2 * l2, dtype=torch.uint8, device=dev)
+    g_ms = []
+    for i in range(20):
+        with torch.cuda.stream(s_gae):
+            flush.fill_(i)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_gae(rewards, store[0].values, dones, store[1].values[0], cfg.gamma, cfg.lam, T, N,
+                    store[0].adv, store[0].ret, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        g_ms.append(a.elapsed_time(b))
+    gae_us = 1e3 * float(np.median(g_ms[3:]))
+    gae_bytes = 17 * T * N + 4 * N
+    # GAE on a widened shape (same T and laws, N = 2^20): the kernel's HBM asymptote
+    Nw = 1 << 20
+    rw, vw, dw, bw = (torch.from_numpy(x).to(dev) for x in wl.make_rollout(cfg, T=T, N=Nw))
+    aw, qw = torch.empty_like(vw), torch.empty_like(vw)
+    w_ms = []
+    for i in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_gae(rw, vw, dw, bw, cfg.gamma, cfg.lam, T, Nw, aw, qw, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        w_ms.append(a.elapsed_time(b))
+    wide_ms = float(np.median(w_ms[3:]))
+    wide_gbs = (17 * T * Nw + 4 * Nw) / (wide_ms * 1e-3) / 1e9
+    del rw, vw, dw, bw, aw, qw
+
+    # ---- dominant kernel and its roofline
+    macs = layer_macs(cfg)
+    top = max(kern, key=lambda k: kern[k]["ms_total"])
+    top_us = kern[top]["us_per_launch"]
+    achieved_tf = 2.0 * macs[top] * N / (top_us * 1e-6) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": achieved_tf / peak_tf, "peak_kind": peak_kind + " sustained", "traffic": None,
+                "us_per_launch": top_us}
+    whole_tf = 2.0 * macs_per_env_step(cfg) * value / world / 1e12
+
+    # ---- end to end through the host-buffer entry points
+    if rank == 0 or dist is not None:
+        h_act = torch.empty(T, N, dtype=torch.int32).pin_memory()
+        h_logp, h_val, h_ent, h_adv, h_ret = (torch.empty(T, N, dtype=torch.float32).pin_memory() for _ in range(5))
+        h_ids = env_ids.cpu().pin_memory()
+        h_rew, h_done = torch.from_numpy(r_np).pin_memory(), torch.from_numpy(d_np).pin_memory()
+        h_boot = torch.zeros(N, dtype=torch.float32).pin_memory()
+
+        def e2e_rollout(k):
+            for t in range(T):
+                hts.hts_policy_step_host(ctx, obs_host[(k * T + t) % ring], h_ids, None, t, SEED + k, N,
+                                         h_act[t], h_logp[t], h_val[t], h_ent[t], None, s_act)
+            hts.hts_gae_host(h_rew, h_val, h_done, h_boot, cfg.gamma, cfg.lam, T, N, h_adv, h_ret, s_act)
+        e2e_rollout(0)
+        barrier()
+        ksteps = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        for k in range(ksteps):
+            e2e_rollout(k + 1)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if dist is not None:
+            ts = torch.tensor([e2e_s], device=dev); dist.all_reduce(ts, op=dist.ReduceOp.MAX); e2e_s = float(ts.item())
+        e2e = {"value": world * ksteps * T * N / e2e_s, "unit": UNIT,
+               "h2d_bytes_per_step": T * (N * obs_bytes + 4 * N) + 9 * T * N + 4 * N,
+               "d2h_bytes_per_step": T * N * 16 + 8 * T * N, "steps": ksteps}
+    hts.hts_policy_destroy(ctx)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- the oracle on this host's cores, bounded sample
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import hts_oracle as orc
+        wt = orc.Weights(params)
+        rows, nsteps = 1024, 8
+        ids = np.arange(rows, dtype=np.int32)
+        t0 = time.perf_counter()
+        for i in range(nsteps):
+            orc.policy_step(wt, obs_host[i % ring].numpy()[:rows], ids, i, SEED)
+        ta = time.perf_counter() - t0
+        rr, vv, dd, bb = wl.make_rollout(cfg)
+        t0 = time.perf_counter()
+        orc.gae(rr, vv, dd, bb, cfg.gamma, cfg.lam)
+        tg = time.perf_counter() - t0
+        cpu = {"value": 1.0 / (ta / (rows * nsteps) + tg / (T * N)), "unit": UNIT, "cores": orc.num_threads(),
+               "kind": "oracle",
+               "sample": f"{nsteps} actor steps x {rows} envs ({ta:.1f} s) + one full GAE [{T},{N}] ({tg*1e3:.1f} ms)"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "N": N, "T": T, "obs": [cfg.C, cfg.H, cfg.W], "actions": A,
+                   "envs_per_gpu": N, "l2": f"observation ring of {ring} batches ({ring * N * obs_bytes >> 20} MiB) exceeds L2 "
+                   f"({l2 >> 20} MiB); GAE-alone timing flushes L2 between launches",
+                   "kernel_times": "second pass over the same rollouts with CUDA events around each kernel"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline,
+        "whole_step_tflops": whole_tf, "whole_step_frac_of_bf16_sustained": whole_tf / peak_tf,
+        "kernels": kern,
+        "gae": {"us_cold": gae_us, "elems_per_s": T * N / (gae_us * 1e-6), "gbs_cold": gae_bytes / (gae_us * 1e-6) / 1e9,
+                "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
+                         "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -131,6 +131,17 @@ hts_status hts_action_uniforms(const int32_t *env_ids, const int32_t *t_per_env,
                                uint64_t seed, int32_t n, int32_t num_actions, float *out,
                                void *cuda_stream);
 
+/* Benchmark support: per-kernel device timing of the actor step.  While enabled, every
+ * hts_policy_step on this context brackets each of its kernels with CUDA events on the
+ * step's stream (up to 4096 steps between two reads; later ones are not recorded).
+ * hts_policy_profile(ctx, 1) starts a fresh collection, (ctx, 0) stops recording.
+ * hts_policy_profile_read waits for the recorded events and returns, for kernel index
+ * 0..4 (hts_policy_kernel_name gives "conv1","conv2","conv3","fc","heads"), the summed
+ * device time in milliseconds and the number of launches recorded.                  */
+hts_status hts_policy_profile(hts_ctx *ctx, int32_t enable);
+hts_status hts_policy_profile_read(hts_ctx *ctx, int32_t kernel, float *total_ms, int32_t *launches);
+const char *hts_policy_kernel_name(int32_t kernel);
+
 /* Reads and clears the device status word of the context (set by a bounded wait
  * that ran out).  Synchronises with the device.  HTS_OK if nothing was recorded.  */
 hts_status hts_last_async_error(hts_ctx *ctx);

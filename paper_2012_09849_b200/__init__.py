@@ -23,7 +23,8 @@ STATUS_NAMES = ["HTS_OK", "HTS_ERR_INVALID_ARG", "HTS_ERR_SHAPE", "HTS_ERR_ALLOC
 WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
                 "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
 EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_host",
-           "hts_policy_read_activation", "hts_action_uniforms", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
+           "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
+           "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
            "hts_gae_host", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
 
 
@@ -67,6 +68,12 @@ def lib():
         L.hts_policy_step_host.argtypes = step
         L.hts_policy_read_activation.argtypes = [vp, i32, i32, vp, vp]
         L.hts_action_uniforms.argtypes = [vp, vp, i32, u64, i32, i32, vp, vp]
+        L.hts_policy_profile.argtypes = [vp, i32]
+        L.hts_policy_profile.restype = C.c_int
+        L.hts_policy_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]
+        L.hts_policy_profile_read.restype = C.c_int
+        L.hts_policy_kernel_name.argtypes = [i32]
+        L.hts_policy_kernel_name.restype = C.c_char_p
         L.hts_last_async_error.argtypes = [vp]
         L.hts_policy_destroy.argtypes = [vp]
         L.hts_policy_destroy.restype = None
@@ -146,6 +153,21 @@ def hts_policy_read_activation(ctx, layer: int, n: int, out, stream=None) -> Non
 def hts_action_uniforms(env_ids, t_per_env, t, seed, n, num_actions, out, stream=None) -> None:
     _check(lib().hts_action_uniforms(_ptr(env_ids), _ptr(t_per_env), int(t), int(seed), int(n), int(num_actions),
                                      _ptr(out), _stream(stream)), "hts_action_uniforms")
+
+
+def hts_policy_profile(ctx, enable: bool) -> None:
+    _check(lib().hts_policy_profile(ctx, int(bool(enable))), "hts_policy_profile")
+
+
+def hts_policy_profile_read(ctx, kernel: int):
+    """-> (total milliseconds, launches) of one kernel of the actor step since profiling was enabled."""
+    ms, cnt = C.c_float(), C.c_int32()
+    _check(lib().hts_policy_profile_read(ctx, int(kernel), C.byref(ms), C.byref(cnt)), "hts_policy_profile_read")
+    return ms.value, cnt.value
+
+
+def hts_policy_kernel_name(kernel: int) -> str:
+    return lib().hts_policy_kernel_name(int(kernel)).decode()
 
 
 def hts_last_async_error(ctx) -> int:

@@ -30,6 +30,18 @@ struct Geometry {
     int H1, W1, H2, W2, H3, W3, F;
 };
 
+// ---- optional per-kernel event timing of the actor step (benchmark support) ------------------
+enum KernelId { K_CONV1 = 0, K_CONV2, K_CONV3, K_FC, K_HEADS, K_COUNT };
+struct Profiler {
+    static constexpr int kCap = 4096;            // event pairs per kernel between two reads
+    bool on = false;
+    int used[K_COUNT] = {0, 0, 0, 0, 0};
+    cudaEvent_t* start[K_COUNT] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t* stop[K_COUNT] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    void begin(int k, cudaStream_t s) { if (on && used[k] < kCap) cudaEventRecord(start[k][used[k]], s); }
+    void end(int k, cudaStream_t s) { if (on && used[k] < kCap) { cudaEventRecord(stop[k][used[k]], s); ++used[k]; } }
+};
+
 // ---- the fp32 CUDA-core path (check path; also the fallback arithmetic for bf16 weights) ---
 struct RefWeights {            // fp32 device copies in PyTorch layouts
     float *w1, *b1, *w2, *b2, *w3, *b3, *wfc, *bfc;
@@ -40,7 +52,7 @@ struct RefWorkspace { float *a1, *a2, *a3, *h; };   // NCHW fp32 activations, [n
 hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& src,
                                const RefWeights& dst, cudaStream_t s);
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
-                       const uint8_t* obs, int n, cudaStream_t s);
+                       const uint8_t* obs, int n, Profiler& prof, cudaStream_t s);
 
 // ---- heads + distribution + sampling epilogue (both paths) --------------------------------
 // h_partials: [num_splits][n][512] fp32.  If fc_bias != nullptr the hidden vector is

@@ -35,6 +35,7 @@ struct hts_ctx {
     int32_t *s_ids = nullptr, *s_t = nullptr, *s_act = nullptr;
     float *s_logp = nullptr, *s_val = nullptr, *s_ent = nullptr, *s_logits = nullptr;
     int* status = nullptr;        // device status word
+    Profiler prof;
     void* allocs[64];
     int nalloc = 0;
 };
@@ -83,11 +84,13 @@ hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids, co
                     float* entropy, float* logits, cudaStream_t s)
 {
     const Geometry& g = ctx->g;
-    hts_status st = ref_forward(g, ctx->rw, ctx->rws, obs, n, s);
+    hts_status st = ref_forward(g, ctx->rw, ctx->rws, obs, n, ctx->prof, s);
     if (st != HTS_OK) return st;
+    ctx->prof.begin(K_HEADS, s);
     st = launch_heads(ctx->rws.h, 1, 0, nullptr, ctx->rw.whead, ctx->rw.bhead, g.A, env_ids, t_per_env, t,
                       seed, n, actions, logp, values, entropy, logits, nullptr, s);
     if (st != HTS_OK) return st;
+    ctx->prof.end(K_HEADS, s);
     ctx->last_n = n;
     return HTS_OK;
 }
@@ -228,9 +231,55 @@ hts_status hts_last_async_error(hts_ctx* ctx)
     return HTS_OK;
 }
 
+hts_status hts_policy_profile(hts_ctx* ctx, int32_t enable)
+{
+    if (!ctx) return HTS_ERR_INVALID_ARG;
+    Profiler& p = ctx->prof;
+    if (enable && !p.start[0]) {
+        for (int k = 0; k < K_COUNT; ++k) {
+            p.start[k] = new (std::nothrow) cudaEvent_t[Profiler::kCap]();
+            p.stop[k] = new (std::nothrow) cudaEvent_t[Profiler::kCap]();
+            if (!p.start[k] || !p.stop[k]) return HTS_ERR_ALLOC;
+            for (int i = 0; i < Profiler::kCap; ++i) {
+                HTS_CUDA(cudaEventCreate(&p.start[k][i]));
+                HTS_CUDA(cudaEventCreate(&p.stop[k][i]));
+            }
+        }
+    }
+    if (enable) for (int k = 0; k < K_COUNT; ++k) p.used[k] = 0;
+    p.on = enable != 0;
+    return HTS_OK;
+}
+
+hts_status hts_policy_profile_read(hts_ctx* ctx, int32_t kernel, float* total_ms, int32_t* launches)
+{
+    if (!ctx || !total_ms || !launches || kernel < 0 || kernel >= K_COUNT) return HTS_ERR_INVALID_ARG;
+    Profiler& p = ctx->prof;
+    float sum = 0.f;
+    for (int i = 0; i < p.used[kernel]; ++i) {
+        float ms = 0.f;
+        HTS_CUDA(cudaEventSynchronize(p.stop[kernel][i]));
+        HTS_CUDA(cudaEventElapsedTime(&ms, p.start[kernel][i], p.stop[kernel][i]));
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = p.used[kernel];
+    return HTS_OK;
+}
+
+const char* hts_policy_kernel_name(int32_t kernel)
+{
+    static const char* names[K_COUNT] = {"conv1", "conv2", "conv3", "fc", "heads"};
+    return (kernel >= 0 && kernel < K_COUNT) ? names[kernel] : "";
+}
+
 void hts_policy_destroy(hts_ctx* ctx)
 {
     if (!ctx) return;
+    for (int k = 0; k < K_COUNT; ++k) {
+        if (ctx->prof.start[k]) { for (int i = 0; i < Profiler::kCap; ++i) cudaEventDestroy(ctx->prof.start[k][i]); delete[] ctx->prof.start[k]; }
+        if (ctx->prof.stop[k]) { for (int i = 0; i < Profiler::kCap; ++i) cudaEventDestroy(ctx->prof.stop[k][i]); delete[] ctx->prof.stop[k]; }
+    }
     for (int i = 0; i < ctx->nalloc; ++i) cudaFree(ctx->allocs[i]);
     delete ctx;
 }

@@ -83,20 +83,28 @@ hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& 
 }
 
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
-                       const uint8_t* obs, int n, cudaStream_t s)
+                       const uint8_t* obs, int n, Profiler& prof, cudaStream_t s)
 {
     const int th = 256;
+    prof.begin(K_CONV1, s);
     conv_direct_kernel<uint8_t><<<blocks_for((size_t)n * 32 * g.H1 * g.W1, th), th, 0, s>>>(
         obs, w.w1, w.b1, ws.a1, n, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, 1.0f / 255.0f);
     HTS_LAUNCH_CHECK("conv1_direct");
+    prof.end(K_CONV1, s);
+    prof.begin(K_CONV2, s);
     conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H2 * g.W2, th), th, 0, s>>>(
         ws.a1, w.w2, w.b2, ws.a2, n, 32, g.H1, g.W1, 64, 4, 2, g.H2, g.W2, 1.0f);
     HTS_LAUNCH_CHECK("conv2_direct");
+    prof.end(K_CONV2, s);
+    prof.begin(K_CONV3, s);
     conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H3 * g.W3, th), th, 0, s>>>(
         ws.a2, w.w3, w.b3, ws.a3, n, 64, g.H2, g.W2, 64, 3, 1, g.H3, g.W3, 1.0f);
     HTS_LAUNCH_CHECK("conv3_direct");
+    prof.end(K_CONV3, s);
+    prof.begin(K_FC, s);
     fc_warp_kernel<<<blocks_for((size_t)n * 512 * 32, th), th, 0, s>>>(ws.a3, w.wfc, w.bfc, ws.h, n, g.F, 512);
     HTS_LAUNCH_CHECK("fc_warp");
+    prof.end(K_FC, s);
     return HTS_OK;
 }
 
