@@ -54,6 +54,17 @@ hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& 
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
                        const uint8_t* obs, int n, Profiler& prof, cudaStream_t s);
 
+// ---- the tensor-core path (bf16 weights) -------------------------------------------------------
+struct TcState;
+hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** out,
+                     bool (*alloc)(void* ctx, void** p, size_t bytes), void* alloc_ctx);
+void tc_destroy(TcState* t);
+hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s);
+hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cudaStream_t s);
+hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
+                    int32_t* actions, float* logp, float* values, float* entropy, float* logits, cudaStream_t s);
+hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s);
+
 // ---- heads + distribution + sampling epilogue (both paths) --------------------------------
 // h_partials: [num_splits][n][512] fp32.  If fc_bias != nullptr the hidden vector is
 // relu(fc_bias + sum over splits in index order), else it is h_partials[0] as is.

@@ -28,15 +28,16 @@ struct hts_ctx {
     Geometry g;
     bool loaded = false;
     int last_n = 0;
-    RefWeights rw{};
+    RefWeights rw{};              // fp32 check path (weight_dtype fp32)
     RefWorkspace rws{};
+    TcState* tc = nullptr;        // tensor-core path (weight_dtype bf16)
     // staging for the host-buffer entry point
     uint8_t* s_obs = nullptr;
     int32_t *s_ids = nullptr, *s_t = nullptr, *s_act = nullptr;
     float *s_logp = nullptr, *s_val = nullptr, *s_ent = nullptr, *s_logits = nullptr;
     int* status = nullptr;        // device status word
     Profiler prof;
-    void* allocs[64];
+    void* allocs[96];
     int nalloc = 0;
 };
 
@@ -46,10 +47,18 @@ template <typename T>
 bool dev_alloc(hts_ctx* c, T** p, size_t count)
 {
     void* q = nullptr;
-    if (c->nalloc >= 64) return false;
+    if (c->nalloc >= 96) return false;
     if (cudaMalloc(&q, count * sizeof(T) + 256) != cudaSuccess) { cudaGetLastError(); return false; }
     c->allocs[c->nalloc++] = q;
     *p = static_cast<T*>(q);
+    return true;
+}
+
+bool raw_alloc(void* c, void** p, size_t bytes)
+{
+    uint8_t* q = nullptr;
+    if (!dev_alloc(static_cast<hts_ctx*>(c), &q, bytes)) return false;
+    *p = q;
     return true;
 }
 
@@ -84,11 +93,19 @@ hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids, co
                     float* entropy, float* logits, cudaStream_t s)
 {
     const Geometry& g = ctx->g;
-    hts_status st = ref_forward(g, ctx->rw, ctx->rws, obs, n, ctx->prof, s);
-    if (st != HTS_OK) return st;
-    ctx->prof.begin(K_HEADS, s);
-    st = launch_heads(ctx->rws.h, 1, 0, nullptr, ctx->rw.whead, ctx->rw.bhead, g.A, env_ids, t_per_env, t,
-                      seed, n, actions, logp, values, entropy, logits, nullptr, s);
+    hts_status st;
+    if (ctx->tc) {
+        st = tc_forward(ctx->tc, obs, n, ctx->prof, s);
+        if (st != HTS_OK) return st;
+        ctx->prof.begin(K_HEADS, s);
+        st = tc_heads(ctx->tc, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy, logits, s);
+    } else {
+        st = ref_forward(g, ctx->rw, ctx->rws, obs, n, ctx->prof, s);
+        if (st != HTS_OK) return st;
+        ctx->prof.begin(K_HEADS, s);
+        st = launch_heads(ctx->rws.h, 1, 0, nullptr, ctx->rw.whead, ctx->rw.bhead, g.A, env_ids, t_per_env, t,
+                          seed, n, actions, logp, values, entropy, logits, nullptr, s);
+    }
     if (st != HTS_OK) return st;
     ctx->prof.end(K_HEADS, s);
     ctx->last_n = n;
@@ -124,18 +141,23 @@ hts_status hts_policy_create(const hts_net_desc* d, hts_ctx** out)
     c->desc = *d; c->g = g;
     const size_t nb = (size_t)d->max_batch;
     const int A = g.A;
-    bool ok = true;
-    ok = ok && dev_alloc(c, &c->rw.w1, (size_t)32 * g.C * 64) && dev_alloc(c, &c->rw.b1, 32);
-    ok = ok && dev_alloc(c, &c->rw.w2, (size_t)64 * 32 * 16) && dev_alloc(c, &c->rw.b2, 64);
-    ok = ok && dev_alloc(c, &c->rw.w3, (size_t)64 * 64 * 9) && dev_alloc(c, &c->rw.b3, 64);
-    ok = ok && dev_alloc(c, &c->rw.wfc, (size_t)512 * g.F) && dev_alloc(c, &c->rw.bfc, 512);
-    ok = ok && dev_alloc(c, &c->rw.whead, (size_t)(A + 1) * 512) && dev_alloc(c, &c->rw.bhead, (size_t)A + 1);
-    ok = ok && dev_alloc(c, &c->rws.a1, nb * 32 * g.H1 * g.W1) && dev_alloc(c, &c->rws.a2, nb * 64 * g.H2 * g.W2);
-    ok = ok && dev_alloc(c, &c->rws.a3, nb * g.F) && dev_alloc(c, &c->rws.h, nb * 512);
+    bool ok = dev_alloc(c, &c->status, 1);
+    if (ok && d->weight_dtype == HTS_DTYPE_BF16) {
+        hts_status st = tc_create(g, d->max_batch, c->status, &c->tc, raw_alloc, c);
+        if (st != HTS_OK) { hts_policy_destroy(c); return st; }
+    } else if (ok) {
+        ok = ok && dev_alloc(c, &c->rw.w1, (size_t)32 * g.C * 64) && dev_alloc(c, &c->rw.b1, 32);
+        ok = ok && dev_alloc(c, &c->rw.w2, (size_t)64 * 32 * 16) && dev_alloc(c, &c->rw.b2, 64);
+        ok = ok && dev_alloc(c, &c->rw.w3, (size_t)64 * 64 * 9) && dev_alloc(c, &c->rw.b3, 64);
+        ok = ok && dev_alloc(c, &c->rw.wfc, (size_t)512 * g.F) && dev_alloc(c, &c->rw.bfc, 512);
+        ok = ok && dev_alloc(c, &c->rw.whead, (size_t)(A + 1) * 512) && dev_alloc(c, &c->rw.bhead, (size_t)A + 1);
+        ok = ok && dev_alloc(c, &c->rws.a1, nb * 32 * g.H1 * g.W1) && dev_alloc(c, &c->rws.a2, nb * 64 * g.H2 * g.W2);
+        ok = ok && dev_alloc(c, &c->rws.a3, nb * g.F) && dev_alloc(c, &c->rws.h, nb * 512);
+    }
     ok = ok && dev_alloc(c, &c->s_obs, nb * g.C * g.H * g.W);
     ok = ok && dev_alloc(c, &c->s_ids, nb) && dev_alloc(c, &c->s_t, nb) && dev_alloc(c, &c->s_act, nb);
     ok = ok && dev_alloc(c, &c->s_logp, nb) && dev_alloc(c, &c->s_val, nb) && dev_alloc(c, &c->s_ent, nb);
-    ok = ok && dev_alloc(c, &c->s_logits, nb * A) && dev_alloc(c, &c->status, 1);
+    ok = ok && dev_alloc(c, &c->s_logits, nb * A);
     if (!ok) { hts_policy_destroy(c); return HTS_ERR_ALLOC; }
     if (cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) {
         hts_status st = cuda_fail(cudaGetLastError(), "cudaMemset");
@@ -152,7 +174,8 @@ hts_status hts_policy_load_weights(hts_ctx* ctx, const hts_weights* w, void* cud
     const void* const* p = reinterpret_cast<const void* const*>(w);
     for (int i = 0; i < 12; ++i) if (!p[i]) return HTS_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    hts_status st = ref_convert_weights(ctx->g, ctx->desc.weight_dtype, *w, ctx->rw, s);
+    hts_status st = ctx->tc ? tc_load_weights(ctx->tc, *w, s)
+                            : ref_convert_weights(ctx->g, ctx->desc.weight_dtype, *w, ctx->rw, s);
     if (st != HTS_OK) return st;
     ctx->loaded = true;
     return HTS_OK;
@@ -204,6 +227,7 @@ hts_status hts_policy_read_activation(hts_ctx* ctx, int32_t layer, int32_t n, fl
     if (!ctx || !out || layer < 1 || layer > 4) return HTS_ERR_INVALID_ARG;
     if (n < 1 || n > ctx->last_n) return HTS_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (ctx->tc) return tc_read_activation(ctx->tc, layer, n, out, s);
     const Geometry& g = ctx->g;
     const float* src = layer == 1 ? ctx->rws.a1 : layer == 2 ? ctx->rws.a2 : layer == 3 ? ctx->rws.a3 : ctx->rws.h;
     const size_t per = layer == 1 ? (size_t)32 * g.H1 * g.W1 : layer == 2 ? (size_t)64 * g.H2 * g.W2
@@ -280,6 +304,7 @@ void hts_policy_destroy(hts_ctx* ctx)
         if (ctx->prof.start[k]) { for (int i = 0; i < Profiler::kCap; ++i) cudaEventDestroy(ctx->prof.start[k][i]); delete[] ctx->prof.start[k]; }
         if (ctx->prof.stop[k]) { for (int i = 0; i < Profiler::kCap; ++i) cudaEventDestroy(ctx->prof.stop[k][i]); delete[] ctx->prof.stop[k]; }
     }
+    if (ctx->tc) tc_destroy(ctx->tc);
     for (int i = 0; i < ctx->nalloc; ++i) cudaFree(ctx->allocs[i]);
     delete ctx;
 }

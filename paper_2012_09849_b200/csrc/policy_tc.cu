@@ -1,0 +1,478 @@
+// Tensor-core path of the actor step (bf16 weights): the convolution and FC layers of the
+// policy-value network (Appendix F.1 / F.2) as tcgen05 GEMMs with TMA-fed shared-memory
+// operands and fp32 accumulators in tensor memory.
+//
+// Formulation.  Activations live in HBM/L2 as row-major [pixel rows, channels] matrices.
+// A k x k / s convolution with k = 2s is a 2x2/1 convolution on the space-to-depth(s) image,
+// and a stride-1 convolution on a flat pixel grid is a sum over taps of row-shifted GEMMs:
+//     D[m, o] = sum_tap sum_c X[m + dy*W_in + dx, c] * W[o, tap, c]
+// computed for every row m of the input grid; rows whose (y, x) fall outside the output extent
+// are discarded by the epilogue.  Every K chunk (64 channels of one tap) is one dense TMA box.
+// The FC layer is the same kernel with one tap and a fixed split of K across CTAs; the split
+// partials are summed in index order by the heads kernel, so nothing depends on the batch size.
+//
+// Operand type.  Both MMA operands are fp16 (kind::f16, fp32 accumulation).  The caller's bf16
+// weights are multiplied by a per-layer power of two that brings the largest magnitude just
+// below 2^15 and converted to fp16: exact for every weight within 2^-29 of the largest (bf16
+// has 8 significant bits, fp16 has 11); the epilogue divides the power of two out again.
+// Activations are stored as fp16 (clamped at the largest finite value): 11 significant bits
+// instead of bf16's 8, which keeps the logits well inside the 2e-2 parity bound.
+#include <new>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace hts {
+using namespace tc;
+
+namespace {
+
+constexpr int BM = 128;                 // rows per tile = TMEM lanes
+constexpr int BK = 64;                  // 16-bit elements per K chunk = one 128-byte swizzle row
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
+enum { EPI_CONV = 0, EPI_SPLITK = 1 };
+enum { L_CONV1 = 0, L_CONV2, L_CONV3, L_FC, L_COUNT };
+
+struct GemmParams {
+    int taps, cpt;                      // filter taps, K chunks per tap
+    int tap_shift[9];                   // row shift of each tap on the flat input grid
+    int nk;                             // K chunks handled by one CTA (all of them, or one split)
+    int n_env;                          // valid environments (conv) / valid rows (FC)
+    int P_in, W_in, H_out, W_out, P_out;   // conv epilogue geometry (pixels per env, grid widths)
+    const float* bias;
+    const float* inv_scale;             // device scalar: undoes the weight scaling of this layer
+    __half* out_h;                      // conv: rows [env*P_out + y*W_out + x][64]
+    float* out_f32;                     // split-K partials [split][rows][ldo]
+    size_t split_stride;
+    int ldo;
+    int* status;
+};
+
+__device__ __forceinline__ uint32_t pack_relu_h2(float a, float b)
+{
+    a = fminf(fmaxf(a, 0.f), 65504.f);
+    b = fminf(fmaxf(b, 0.f), 65504.f);
+    __half2 t = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(192)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p)
+{
+    constexpr int B_BYTES = BN * BK * 2;
+    constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], accum_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kc = 0; kc < p.nk; ++kc) {
+                const int s = kc % STAGES;
+                const uint32_t ph = (uint32_t)(kc / STAGES) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u, abortp, p.status, 1)) break;
+                const int g = blockIdx.z * p.nk + kc;
+                const int tap = g / p.cpt, sub = g - tap * p.cpt;
+                uint8_t* a_dst = tiles + s * STAGE_BYTES;
+                mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+                tma_load_2d(a_dst, &tmA, sub * BK, m0 + p.tap_shift[tap], &full_bar[s]);
+                tma_load_2d(a_dst + A_BYTES, &tmB, g * BK, n0, &full_bar[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_f16(0, BM, BN);
+            for (int kc = 0; kc < p.nk; ++kc) {
+                const int s = kc % STAGES;
+                const uint32_t ph = (uint32_t)(kc / STAGES) & 1u;
+                if (!mbar_wait(&full_bar[s], ph, abortp, p.status, 2)) break;
+                tc_fence_after();
+                const uint32_t a_addr = base + s * STAGE_BYTES;
+                const uint64_t adesc = smem_desc_sw128(a_addr);
+                const uint64_t bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)       // 32 bytes further along the swizzled row per K step
+                    mma_f16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | k) != 0);
+                mma_commit(&empty_bar[s]);
+            }
+            mma_commit(&accum_bar);
+        }
+    } else {
+        // epilogue warps 2..5: warp w may touch TMEM lanes [32*(w%4), 32*(w%4)+32)
+        const int q = warp & 3;
+        const int r = q * 32 + lane;                    // row of the tile = TMEM lane
+        const bool ok = mbar_wait(&accum_bar, 0, abortp, p.status, 3);
+        tc_fence_after();
+        if (ok) {
+            const long m = (long)m0 + r;
+            const float inv = *p.inv_scale;
+            if (EPI == EPI_SPLITK) {
+                float* dst = p.out_f32 + blockIdx.z * p.split_stride + (size_t)m * p.ldo + n0;
+#pragma unroll
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+                    tmem_ld_wait();
+                    if (m < p.n_env) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(dst + c + j) =
+                                make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
+                                            __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                    }
+                }
+            } else {
+                const int env = (int)(m / p.P_in);
+                const int pix = (int)(m - (long)env * p.P_in);
+                const int y = pix / p.W_in, x = pix - y * p.W_in;
+                const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
+                __half* dst = p.out_h + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * BN;
+#pragma unroll
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int h = 0; h < 4; ++h)
+                                pk[h] = pack_relu_h2(fmaf(__uint_as_float(v[j + 2 * h]), inv, p.bias[n0 + c + j + 2 * h]),
+                                                     fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, p.bias[n0 + c + j + 2 * h + 1]));
+                            *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (*abortp) {                                      // give copies still in flight time to land
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_d, TMEM_COLS);
+}
+
+// ---- weight scaling and packing ---------------------------------------------------------------
+__global__ void absmax_kernel(const __nv_bfloat16* __restrict__ w, size_t n, unsigned* __restrict__ slot)
+{
+    unsigned m = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float a = fabsf(__bfloat162float(w[i]));
+        if (a == a && a < INFINITY) m = max(m, __float_as_uint(a));     // finite magnitudes order like their bits
+    }
+    for (int k = 16; k > 0; k >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, k));
+    if ((threadIdx.x & 31) == 0 && m) atomicMax(slot, m);
+}
+// scale = 2^(14 - floor(log2 max)): the largest weight lands in [2^14, 2^15)
+__global__ void scales_kernel(const unsigned* __restrict__ slots, float* __restrict__ scale, float* __restrict__ inv,
+                              float conv1_extra)
+{
+    const int l = threadIdx.x;
+    if (l >= L_COUNT) return;
+    const float mx = __uint_as_float(slots[l]);
+    int e = 0;
+    float s = 1.f;
+    if (mx > 0.f) { frexpf(mx, &e); s = ldexpf(1.f, 15 - e); }        // mx = f * 2^e, f in [0.5, 1)
+    scale[l] = s;
+    inv[l] = (l == L_CONV1 ? conv1_extra : 1.f) / s;
+}
+__device__ __forceinline__ __half scaled_h(__nv_bfloat16 w, float s) { return __float2half_rn(__bfloat162float(w) * s); }
+
+// conv2: Wp[o][(tap*2 + half)*64 + j], c' = half*64 + j = (uy*2+ux)*32 + c, tap = dy*2+dx,
+//        value w2[o][c][2dy+uy][2dx+ux]
+__global__ void pack_conv2_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, const float* __restrict__ scale)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 64 * 512) return;
+    const int o = i / 512, k = i % 512;
+    const int tap = k / 128, cp = k % 128;
+    const int dy = tap >> 1, dx = tap & 1, uy = (cp / 32) >> 1, ux = (cp / 32) & 1, c = cp % 32;
+    wp[i] = scaled_h(w[((o * 32 + c) * 4 + (2 * dy + uy)) * 4 + (2 * dx + ux)], scale[L_CONV2]);
+}
+// conv3: Wp[o][(dy*3+dx)*64 + c] = w3[o][c][dy][dx]
+__global__ void pack_conv3_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, const float* __restrict__ scale)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 64 * 576) return;
+    const int o = i / 576, k = i % 576;
+    const int tap = k / 64, c = k % 64;
+    wp[i] = scaled_h(w[(o * 64 + c) * 9 + tap], scale[L_CONV3]);
+}
+// FC: Wp[o][pix*64 + c] = wfc[o][c*P3 + pix]   (activations are stored pixel-major, channel-minor)
+__global__ void pack_fc_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int P3, const float* __restrict__ scale)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int F = 64 * P3;
+    if (i >= (size_t)512 * F) return;
+    const int o = (int)(i / F), k = (int)(i % F);
+    const int pix = k / 64, c = k % 64;
+    wp[i] = scaled_h(w[(size_t)o * F + c * P3 + pix], scale[L_FC]);
+}
+__global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, size_t n)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = __bfloat162float(src[i]);
+}
+
+// ---- stand-in conv1: CUDA-core direct convolution writing the space-to-depth(2) fp16 layout ------
+__global__ void conv1_direct_s2d_kernel(const uint8_t* __restrict__ x, const float* __restrict__ w,
+                                        const float* __restrict__ b, __half* __restrict__ out,
+                                        int n, int C, int H, int W, int H1, int W1, int P1s, int W1s)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t total = (size_t)n * 32 * H1 * W1;
+    if (idx >= total) return;
+    const int j = (int)(idx % W1);
+    const int i = (int)((idx / W1) % H1);
+    const int o = (int)((idx / ((size_t)W1 * H1)) % 32);
+    const size_t e = idx / ((size_t)W1 * H1 * 32);
+    const uint8_t* xe = x + e * (size_t)C * H * W;
+    const float* wo = w + (size_t)o * C * 64;
+    float acc = 0.f;
+    for (int c = 0; c < C; ++c)
+        for (int u = 0; u < 8; ++u) {
+            const uint8_t* xr = xe + ((size_t)c * H + (i * 4 + u)) * W + j * 4;
+            const float* wr = wo + (c * 8 + u) * 8;
+            for (int v = 0; v < 8; ++v) acc = fmaf(wr[v], (float)xr[v], acc);
+        }
+    acc = fmaf(acc, 1.0f / 255.0f, b[o]);
+    acc = fminf(fmaxf(acc, 0.f), 65504.f);
+    out[(e * P1s + (size_t)(i >> 1) * W1s + (j >> 1)) * 128 + ((i & 1) * 2 + (j & 1)) * 32 + o] = __float2half_rn(acc);
+}
+
+// ---- parity taps: internal layouts -> fp32 NCHW ----------------------------------------------------
+__global__ void tap_rows_kernel(const __half* __restrict__ src, float* __restrict__ dst, int n, int Cc,
+                                int Ho, int Wo, int s2d, int P_rows, int W_rows)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t total = (size_t)n * Cc * Ho * Wo;
+    if (idx >= total) return;
+    const int x = (int)(idx % Wo), y = (int)((idx / Wo) % Ho), c = (int)((idx / ((size_t)Wo * Ho)) % Cc);
+    const size_t e = idx / ((size_t)Wo * Ho * Cc);
+    size_t off;
+    if (s2d) off = (e * P_rows + (size_t)(y >> 1) * W_rows + (x >> 1)) * (4 * Cc) + ((y & 1) * 2 + (x & 1)) * Cc + c;
+    else off = (e * P_rows + (size_t)y * W_rows + x) * Cc + c;
+    dst[idx] = __half2float(src[off]);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D fp16 row-major [rows, cols] matrix, box [box_rows x 64 cols], 128-byte swizzle, zero fill.
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch_bytes};
+    const cuuint32_t box[2] = {BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline unsigned nblk(size_t total, int th) { return (unsigned)((total + th - 1) / th); }
+
+template <int BN, int EPI>
+hts_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, dim3 grid, cudaStream_t s)
+{
+    constexpr int smem = STAGES * (A_BYTES + BN * BK * 2) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_set = true;
+    }
+    gemm_tc_kernel<BN, EPI><<<grid, 192, smem, s>>>(a, b, p);
+    HTS_LAUNCH_CHECK("gemm_tc_kernel");
+    return HTS_OK;
+}
+
+}  // namespace
+
+struct TcState {
+    Geometry g;
+    int max_batch;
+    int H1s, W1s, P1s;          // space-to-depth(2) grid of the conv1 output
+    int P2, P3;
+    int splits, cps;            // FC split-K
+    // packed weights
+    __half *w2p, *w3p, *wfcp;
+    float *w1f, *b1, *b2, *b3, *bfc, *whead, *bhead;
+    unsigned* absmax;           // [L_COUNT]
+    float *scale, *inv_scale;   // [L_COUNT] each
+    // workspace
+    __half *a1s, *a2, *a3;
+    float *hpart, *h;
+    CUtensorMap mA2, mB2, mA3, mB3, mAfc, mBfc;
+    int* status;
+};
+
+hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** out,
+                     bool (*alloc)(void* ctx, void** p, size_t bytes), void* alloc_ctx)
+{
+    TcState* t = new (std::nothrow) TcState();
+    if (!t) return HTS_ERR_ALLOC;
+    t->g = g; t->max_batch = max_batch; t->status = status;
+    t->H1s = (g.H1 + 1) / 2; t->W1s = (g.W1 + 1) / 2; t->P1s = t->H1s * t->W1s;
+    t->P2 = g.H2 * g.W2; t->P3 = g.H3 * g.W3;
+    const int chunks = g.F / BK;
+    t->splits = 1;
+    for (int s = 8; s >= 1; --s) if (chunks % s == 0) { t->splits = s; break; }
+    t->cps = chunks / t->splits;
+    const size_t nb = (size_t)max_batch;
+    auto A = [&](auto** p, size_t count) { return alloc(alloc_ctx, reinterpret_cast<void**>(p), count * sizeof(**p)); };
+    bool ok = A(&t->w2p, (size_t)64 * 512) && A(&t->w3p, (size_t)64 * 576) && A(&t->wfcp, (size_t)512 * g.F) &&
+              A(&t->w1f, (size_t)32 * g.C * 64) && A(&t->b1, 32) && A(&t->b2, 64) && A(&t->b3, 64) && A(&t->bfc, 512) &&
+              A(&t->whead, (size_t)(g.A + 1) * 512) && A(&t->bhead, (size_t)g.A + 1) &&
+              A(&t->absmax, L_COUNT) && A(&t->scale, L_COUNT) && A(&t->inv_scale, L_COUNT) &&
+              A(&t->a1s, nb * t->P1s * 128) && A(&t->a2, nb * t->P2 * 64) && A(&t->a3, nb * g.F) &&
+              A(&t->hpart, (size_t)t->splits * nb * 512) && A(&t->h, nb * 512);
+    if (!ok) { delete t; return HTS_ERR_ALLOC; }
+    // cells of an odd-sized s2d border that conv1 never writes must hold finite numbers
+    if (cudaMemset(t->a1s, 0, nb * t->P1s * 128 * 2) != cudaSuccess) { delete t; return cuda_fail(cudaGetLastError(), "cudaMemset"); }
+    ok = make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, BM) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
+         make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, BM) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
+         make_map(&t->mAfc, t->a3, nb, g.F, (uint64_t)g.F * 2, BM) && make_map(&t->mBfc, t->wfcp, 512, g.F, (uint64_t)g.F * 2, 128);
+    if (!ok) { delete t; return HTS_ERR_CUDA; }
+    *out = t;
+    return HTS_OK;
+}
+
+void tc_destroy(TcState* t) { delete t; }
+
+hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s)
+{
+    const Geometry& g = t->g;
+    auto bf = [](const void* p) { return static_cast<const __nv_bfloat16*>(p); };
+    HTS_CUDA(cudaMemsetAsync(t->absmax, 0, L_COUNT * sizeof(unsigned), s));
+    struct Mx { const void* p; size_t n; int l; };
+    const Mx mx[] = {{w.conv1_w, (size_t)32 * g.C * 64, L_CONV1}, {w.conv2_w, (size_t)64 * 512, L_CONV2},
+                     {w.conv3_w, (size_t)64 * 576, L_CONV3}, {w.fc_w, (size_t)512 * g.F, L_FC}};
+    for (const Mx& m : mx) {
+        absmax_kernel<<<64, 256, 0, s>>>(bf(m.p), m.n, t->absmax + m.l);
+        HTS_LAUNCH_CHECK("absmax");
+    }
+    scales_kernel<<<1, 32, 0, s>>>(t->absmax, t->scale, t->inv_scale, 1.0f / 255.0f);
+    HTS_LAUNCH_CHECK("scales");
+    pack_conv2_kernel<<<nblk(64 * 512, 256), 256, 0, s>>>(bf(w.conv2_w), t->w2p, t->scale); HTS_LAUNCH_CHECK("pack_conv2");
+    pack_conv3_kernel<<<nblk(64 * 576, 256), 256, 0, s>>>(bf(w.conv3_w), t->w3p, t->scale); HTS_LAUNCH_CHECK("pack_conv3");
+    pack_fc_kernel<<<nblk((size_t)512 * g.F, 256), 256, 0, s>>>(bf(w.fc_w), t->wfcp, t->P3, t->scale); HTS_LAUNCH_CHECK("pack_fc");
+    struct It { const void* p; float* q; size_t n; };
+    const It items[] = {{w.conv1_w, t->w1f, (size_t)32 * g.C * 64}, {w.conv1_b, t->b1, 32}, {w.conv2_b, t->b2, 64},
+                        {w.conv3_b, t->b3, 64}, {w.fc_b, t->bfc, 512}, {w.pi_w, t->whead, (size_t)g.A * 512},
+                        {w.v_w, t->whead + (size_t)g.A * 512, 512}, {w.pi_b, t->bhead, (size_t)g.A}, {w.v_b, t->bhead + g.A, 1}};
+    for (const It& it : items) {
+        bf16_to_f32_kernel<<<nblk(it.n, 256), 256, 0, s>>>(bf(it.p), it.q, it.n);
+        HTS_LAUNCH_CHECK("bf16_to_f32");
+    }
+    return HTS_OK;
+}
+
+hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cudaStream_t s)
+{
+    const Geometry& g = t->g;
+    prof.begin(K_CONV1, s);
+    conv1_direct_s2d_kernel<<<nblk((size_t)n * 32 * g.H1 * g.W1, 256), 256, 0, s>>>(
+        obs, t->w1f, t->b1, t->a1s, n, g.C, g.H, g.W, g.H1, g.W1, t->P1s, t->W1s);
+    HTS_LAUNCH_CHECK("conv1_direct_s2d");
+    prof.end(K_CONV1, s);
+
+    GemmParams p{};
+    p.status = t->status; p.n_env = n;
+    // conv2: 2x2 taps on the s2d grid [H1s, W1s] with 128 channels -> [H2, W2] x 64
+    p.taps = 4; p.cpt = 2; p.nk = 8;
+    p.tap_shift[0] = 0; p.tap_shift[1] = 1; p.tap_shift[2] = t->W1s; p.tap_shift[3] = t->W1s + 1;
+    p.P_in = t->P1s; p.W_in = t->W1s; p.H_out = g.H2; p.W_out = g.W2; p.P_out = t->P2;
+    p.bias = t->b2; p.out_h = t->a2; p.inv_scale = t->inv_scale + L_CONV2;
+    prof.begin(K_CONV2, s);
+    hts_status st = launch_gemm<64, EPI_CONV>(t->mA2, t->mB2, p, dim3(nblk((size_t)n * t->P1s, BM), 1, 1), s);
+    if (st != HTS_OK) return st;
+    prof.end(K_CONV2, s);
+    // conv3: 3x3 taps on [H2, W2] x 64 -> [H3, W3] x 64
+    p.taps = 9; p.cpt = 1; p.nk = 9;
+    for (int dy = 0; dy < 3; ++dy) for (int dx = 0; dx < 3; ++dx) p.tap_shift[dy * 3 + dx] = dy * g.W2 + dx;
+    p.P_in = t->P2; p.W_in = g.W2; p.H_out = g.H3; p.W_out = g.W3; p.P_out = t->P3;
+    p.bias = t->b3; p.out_h = t->a3; p.inv_scale = t->inv_scale + L_CONV3;
+    prof.begin(K_CONV3, s);
+    st = launch_gemm<64, EPI_CONV>(t->mA3, t->mB3, p, dim3(nblk((size_t)n * t->P2, BM), 1, 1), s);
+    if (st != HTS_OK) return st;
+    prof.end(K_CONV3, s);
+    // FC: [n, F] x [512, F]^T, K split across blockIdx.z
+    p.taps = 1; p.cpt = g.F / BK; p.nk = t->cps; p.tap_shift[0] = 0;
+    p.out_f32 = t->hpart; p.split_stride = (size_t)t->max_batch * 512; p.ldo = 512; p.inv_scale = t->inv_scale + L_FC;
+    prof.begin(K_FC, s);
+    st = launch_gemm<128, EPI_SPLITK>(t->mAfc, t->mBfc, p, dim3(nblk(n, BM), 4, t->splits), s);
+    if (st != HTS_OK) return st;
+    prof.end(K_FC, s);
+    return HTS_OK;
+}
+
+hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
+                    int32_t* actions, float* logp, float* values, float* entropy, float* logits, cudaStream_t s)
+{
+    return launch_heads(t->hpart, t->splits, (size_t)t->max_batch * 512, t->bfc, t->whead, t->bhead, t->g.A, env_ids,
+                        t_per_env, tt, seed, n, actions, logp, values, entropy, logits, t->h, s);
+}
+
+hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s)
+{
+    const Geometry& g = t->g;
+    if (layer == 4) {
+        HTS_CUDA(cudaMemcpyAsync(out, t->h, (size_t)n * 512 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        return HTS_OK;
+    }
+    if (layer == 1)
+        tap_rows_kernel<<<nblk((size_t)n * 32 * g.H1 * g.W1, 256), 256, 0, s>>>(t->a1s, out, n, 32, g.H1, g.W1, 1, t->P1s, t->W1s);
+    else if (layer == 2)
+        tap_rows_kernel<<<nblk((size_t)n * 64 * g.H2 * g.W2, 256), 256, 0, s>>>(t->a2, out, n, 64, g.H2, g.W2, 0, t->P2, g.W2);
+    else
+        tap_rows_kernel<<<nblk((size_t)n * 64 * g.H3 * g.W3, 256), 256, 0, s>>>(t->a3, out, n, 64, g.H3, g.W3, 0, t->P3, g.W3);
+    HTS_LAUNCH_CHECK("tap_rows_kernel");
+    return HTS_OK;
+}
+
+}  // namespace hts
