@@ -1,0 +1,277 @@
+// conv1 (8x8 / 4, C -> 32) of the policy-value network, fused from raw frames to fp16 output.
+//
+// An 8x8 stride-4 convolution is a 2x2 stride-1 convolution on the space-to-depth(4) image
+// (channels c' = c*16 + uy*4 + ux).  One work unit is a band of R output rows of one
+// environment: its (R+1) x Ws space-to-depth pixels become the rows of an fp16 tile in shared
+// memory (128-byte swizzled rows of 64 channels, one plane per 64 channels), and each filter tap
+// (dy,dx) is the same tile read from a start address shifted by dy*Ws+dx rows.  Output row
+// m = y*Ws + x of the 128-row MMA tile is pixel (y, x) of the band; x = Ws-1 and rows past the
+// band are computed and thrown away.
+//
+// Stages per unit: bulk copies (cp.async.bulk, one per channel) bring the band's uint8 rows
+// into a two-deep ring; four warps convert them to fp16 (bytes 0..255 are exact in fp16; the
+// 1/255 is folded into the accumulator scale) and write the tile; one thread issues
+// 16 * planes tcgen05.mma (128 x 32 x 16) into tensor memory; the same four warps read the
+// accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
+#include "conv1_tc.cuh"
+#include "tc_ptx.cuh"
+
+namespace hts {
+using namespace tc;
+
+namespace {
+
+constexpr int kThreads = 160;                   // warp 0: copies + MMA issue, warps 1..4: convert + epilogue
+constexpr int kWorkers = 128;
+constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x 128 bytes
+
+struct Conv1Params {
+    Conv1Plan pl;
+    const uint8_t* obs;
+    int n;
+    const float* bias;
+    const float* inv_scale;
+    __half* out;
+    int* status;
+};
+
+// four bytes -> four fp16 values (b0,b1 | b2,b3), exact: 0x64xx is 1024 + xx
+__device__ __forceinline__ void u8x4_to_h4(uint32_t w, uint32_t& lo, uint32_t& hi)
+{
+    const uint32_t magic = 0x64646464u;
+    uint32_t a = __byte_perm(w, magic, 0x4140);         // {b0, 0x64, b1, 0x64} as two halves 0x64b0, 0x64b1
+    uint32_t b = __byte_perm(w, magic, 0x4342);
+    const __half2 k = __half2half2(__ushort_as_half((unsigned short)0x6400));
+    __half2 ha = __hsub2(*reinterpret_cast<__half2*>(&a), k);
+    __half2 hb = __hsub2(*reinterpret_cast<__half2*>(&b), k);
+    lo = *reinterpret_cast<uint32_t*>(&ha);
+    hi = *reinterpret_cast<uint32_t*>(&hb);
+}
+
+__global__ void __launch_bounds__(kThreads)
+conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
+{
+    const Conv1Plan& pl = p.pl;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t w_bar, u8_full[2], u8_empty[2], a_ready, d_full;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    volatile int* abortp = &abort_flag;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    const int plane_bytes = pl.tile_rows * 128;
+    const int w_bytes = 4 * pl.cpt * kChunkBytes;
+    // layout: [weights][fp16 tile: cpt planes][u8 stage 0][u8 stage 1]
+    uint8_t* s_w = sm;
+    uint8_t* s_tile = sm + w_bytes;
+    uint8_t* s_u8 = s_tile + pl.cpt * plane_bytes;
+    const uint32_t a_w = base, a_tile = base + w_bytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int units = p.n * pl.bands;
+    const int band_in_rows = 4 * (pl.R + 1);
+
+    if (threadIdx.x == 0) {
+        mbar_init(&w_bar, 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kWorkers); }
+        mbar_init(&a_ready, kWorkers);
+        mbar_init(&d_full, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmW);
+    }
+    if (warp == 0) tmem_alloc(&tmem_slot, 32);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // weights once
+            mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
+            for (int g = 0; g < 4 * pl.cpt; ++g) tma_load_2d(s_w + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+            constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
+            bool alive = true;
+            // software pipeline: the copy of unit i+1 is issued before the MMAs of unit i
+            auto issue_copy = [&](int it, int u) -> bool {
+                const int s = it & 1;
+                if (!mbar_wait(&u8_empty[s], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 11)) return false;
+                const int env = u / pl.bands, band = u - env * pl.bands;
+                const int r0 = 4 * band * pl.R;
+                int rows = pl.H - r0; rows = rows > band_in_rows ? band_in_rows : rows;
+                const uint32_t bytes = (uint32_t)(rows * pl.W);
+                mbar_arrive_expect_tx(&u8_full[s], bytes * pl.C);
+                const uint8_t* src = p.obs + ((size_t)env * pl.C * pl.H + r0) * pl.W;
+                uint8_t* dst = s_u8 + s * pl.u8_stage_bytes;
+                for (int c = 0; c < pl.C; ++c)
+                    bulk_load(dst + c * band_in_rows * pl.W, src + (size_t)c * pl.H * pl.W, bytes, &u8_full[s]);
+                return true;
+            };
+            int it = 0;
+            int u = blockIdx.x;
+            if (u < units) alive = issue_copy(0, u);
+            if (alive) alive = mbar_wait(&w_bar, 0, abortp, p.status, 12);
+            for (; alive && u < units; u += gridDim.x, ++it) {
+                const int un = u + gridDim.x;
+                if (un < units) { if (!issue_copy(it + 1, un)) break; }
+                if (!mbar_wait(&a_ready, (uint32_t)it & 1u, abortp, p.status, 13)) break;
+                tc_fence_after();
+                uint32_t first = 1;
+                for (int tap = 0; tap < 4; ++tap) {
+                    const int shift = (tap >> 1) * pl.Ws + (tap & 1);
+                    for (int pln = 0; pln < pl.cpt; ++pln) {
+                        const uint64_t adesc = smem_desc_sw128(a_tile + pln * plane_bytes + shift * 128);
+                        const uint64_t bdesc = smem_desc_sw128(a_w + (tap * pl.cpt + pln) * kChunkBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            mma_f16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, first ? 0u : 1u);
+                            first = 0;
+                        }
+                    }
+                }
+                mma_commit(&d_full);
+            }
+        }
+    } else {
+        const int tid = threadIdx.x - 32;                // 0..127
+        const int q = warp & 3;                          // TMEM lane quarter this warp may read
+        const int row = q * 32 + lane;                   // tile row handled in the epilogue
+        const float inv = *p.inv_scale;
+        float bias[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) bias[j] = p.bias[j];
+        int it = 0;
+        for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
+            const int s = it & 1;
+            const int env = u / pl.bands, band = u - env * pl.bands;
+            const int y0 = band * pl.R;
+            int in_rows = pl.H - 4 * y0; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
+            const int s2d_rows = in_rows >> 2;           // space-to-depth rows present in this band
+            if (!mbar_wait(&u8_full[s], ((uint32_t)it >> 1) & 1u, abortp, p.status, 14)) break;
+            // ---- convert: item = (plane, pixel, 16-byte chunk): 2 rows x 4 bytes of one channel
+            const uint8_t* src = s_u8 + s * pl.u8_stage_bytes;
+            const int pixels = s2d_rows * pl.Ws;
+            const int items = pl.cpt * pixels * 8;
+            for (int i = tid; i < items; i += kWorkers) {
+                const int qq = i & 7;
+                const int rest = i >> 3;
+                const int pln = rest / pixels;
+                const int ps = rest - pln * pixels;
+                const int ys = ps / pl.Ws, xs = ps - ys * pl.Ws;
+                const int c = pln * 4 + (qq >> 1);
+                const uint8_t* s0 = src + (c * band_in_rows + 4 * ys + 2 * (qq & 1)) * pl.W + 4 * xs;
+                const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
+                const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
+                uint4 o;
+                u8x4_to_h4(w0, o.x, o.y);
+                u8x4_to_h4(w1, o.z, o.w);
+                *reinterpret_cast<uint4*>(s_tile + pln * plane_bytes + ps * 128 + ((qq ^ (ps & 7)) << 4)) = o;
+            }
+            fence_async_proxy();                         // tile stores -> visible to the tensor core's reads
+            mbar_arrive(&u8_empty[s]);
+            mbar_arrive(&a_ready);
+            // ---- epilogue
+            if (!mbar_wait(&d_full, (uint32_t)it & 1u, abortp, p.status, 15)) break;
+            tc_fence_after();
+            uint32_t v[32];
+            tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16), v);
+            tmem_ld_wait();
+            tc_fence_before();
+            const int y = row / pl.Ws, x = row - y * pl.Ws;
+            const int yy = y0 + y;
+            if (y < pl.R && yy < pl.H1 && x < pl.W1) {
+                __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (x >> 1)) * 128 +
+                              ((yy & 1) * 2 + (x & 1)) * 32;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        float a = fmaf(__uint_as_float(v[j + 2 * h]), inv, bias[j + 2 * h]);
+                        float b = fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, bias[j + 2 * h + 1]);
+                        a = fminf(fmaxf(a, 0.f), 65504.f);
+                        b = fminf(fmaxf(b, 0.f), 65504.f);
+                        __half2 t = __floats2half2_rn(a, b);
+                        pk[h] = *reinterpret_cast<uint32_t*>(&t);
+                    }
+                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+        }
+    }
+    if (*abortp) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_d, 32);
+}
+
+__global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int C,
+                                  const float* __restrict__ scale)
+{
+    const int Cs = 16 * C;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 32 * 4 * Cs) return;
+    const int o = i / (4 * Cs), k = i % (4 * Cs);
+    const int tap = k / Cs, cp = k % Cs;
+    const int dy = tap >> 1, dx = tap & 1, c = cp >> 4, uy = (cp >> 2) & 3, ux = cp & 3;
+    wp[i] = __float2half_rn(__bfloat162float(w[((o * C + c) * 8 + (4 * dy + uy)) * 8 + (4 * dx + ux)]) * scale[0]);
+}
+
+}  // namespace
+
+bool conv1_plan(const Geometry& g, Conv1Plan* pl)
+{
+    if (g.C % 4 || g.H % 4 || g.W % 4) return false;    // bulk copies then start and end on 16-byte boundaries
+    pl->C = g.C; pl->H = g.H; pl->W = g.W;
+    pl->Hs = g.H / 4; pl->Ws = g.W / 4; pl->Cs = 16 * g.C;
+    pl->H1 = pl->Hs - 1; pl->W1 = pl->Ws - 1;
+    if (pl->H1 != g.H1 || pl->W1 != g.W1 || pl->Ws > 64 || pl->H1 < 1) return false;
+    pl->cpt = pl->Cs / 64;
+    const int rmax = 128 / pl->Ws;
+    pl->bands = (pl->H1 + rmax - 1) / rmax;
+    pl->R = (pl->H1 + pl->bands - 1) / pl->bands;
+    pl->tile_rows = (128 + pl->Ws + 1 + 7) / 8 * 8;
+    pl->u8_stage_bytes = (g.C * 4 * (pl->R + 1) * g.W + 127) / 128 * 128;
+    pl->smem_bytes = 1024 + 4 * pl->cpt * kChunkBytes + pl->cpt * pl->tile_rows * 128 + 2 * pl->u8_stage_bytes;
+    pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
+    return pl->smem_bytes <= 227 * 1024;
+}
+
+hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __half* packed, const float* scale,
+                              cudaStream_t s)
+{
+    const int total = 32 * 4 * pl.Cs;
+    pack_conv1_kernel<<<(total + 255) / 256, 256, 0, s>>>(w1, packed, pl.C, scale);
+    HTS_LAUNCH_CHECK("pack_conv1");
+    return HTS_OK;
+}
+
+hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, int n,
+                        const float* bias, const float* inv_scale, __half* out, int* status, cudaStream_t s)
+{
+    static int sm_count = 0, max_smem_set = 0;
+    if (!sm_count) {
+        int dev = 0;
+        HTS_CUDA(cudaGetDevice(&dev));
+        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if (max_smem_set < pl.smem_bytes) {
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
+        max_smem_set = pl.smem_bytes;
+    }
+    const int per_sm = (227 * 1024) / (pl.smem_bytes + 1024) > 4 ? 4 : (227 * 1024) / (pl.smem_bytes + 1024);
+    const int units = n * pl.bands;
+    int grid = sm_count * (per_sm < 1 ? 1 : per_sm);
+    if (grid > units) grid = units;
+    Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
+    conv1_tc_kernel<<<grid, kThreads, pl.smem_bytes, s>>>(weight_map, p);
+    HTS_LAUNCH_CHECK("conv1_tc_kernel");
+    return HTS_OK;
+}
+
+}  // namespace hts

@@ -22,6 +22,8 @@
 #include <cuda_fp16.h>
 #include "common.cuh"
 #include "tc_ptx.cuh"
+#include "tc_host.cuh"
+#include "conv1_tc.cuh"
 
 namespace hts {
 using namespace tc;
@@ -243,32 +245,6 @@ __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ src, float*
     if (i < n) dst[i] = __bfloat162float(src[i]);
 }
 
-// ---- stand-in conv1: CUDA-core direct convolution writing the space-to-depth(2) fp16 layout ------
-__global__ void conv1_direct_s2d_kernel(const uint8_t* __restrict__ x, const float* __restrict__ w,
-                                        const float* __restrict__ b, __half* __restrict__ out,
-                                        int n, int C, int H, int W, int H1, int W1, int P1s, int W1s)
-{
-    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const size_t total = (size_t)n * 32 * H1 * W1;
-    if (idx >= total) return;
-    const int j = (int)(idx % W1);
-    const int i = (int)((idx / W1) % H1);
-    const int o = (int)((idx / ((size_t)W1 * H1)) % 32);
-    const size_t e = idx / ((size_t)W1 * H1 * 32);
-    const uint8_t* xe = x + e * (size_t)C * H * W;
-    const float* wo = w + (size_t)o * C * 64;
-    float acc = 0.f;
-    for (int c = 0; c < C; ++c)
-        for (int u = 0; u < 8; ++u) {
-            const uint8_t* xr = xe + ((size_t)c * H + (i * 4 + u)) * W + j * 4;
-            const float* wr = wo + (c * 8 + u) * 8;
-            for (int v = 0; v < 8; ++v) acc = fmaf(wr[v], (float)xr[v], acc);
-        }
-    acc = fmaf(acc, 1.0f / 255.0f, b[o]);
-    acc = fminf(fmaxf(acc, 0.f), 65504.f);
-    out[(e * P1s + (size_t)(i >> 1) * W1s + (j >> 1)) * 128 + ((i & 1) * 2 + (j & 1)) * 32 + o] = __float2half_rn(acc);
-}
-
 // ---- parity taps: internal layouts -> fp32 NCHW ----------------------------------------------------
 __global__ void tap_rows_kernel(const __half* __restrict__ src, float* __restrict__ dst, int n, int Cc,
                                 int Ho, int Wo, int s2d, int P_rows, int W_rows)
@@ -282,37 +258,6 @@ __global__ void tap_rows_kernel(const __half* __restrict__ src, float* __restric
     if (s2d) off = (e * P_rows + (size_t)(y >> 1) * W_rows + (x >> 1)) * (4 * Cc) + ((y & 1) * 2 + (x & 1)) * Cc + c;
     else off = (e * P_rows + (size_t)y * W_rows + x) * Cc + c;
     dst[idx] = __half2float(src[off]);
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// 2-D fp16 row-major [rows, cols] matrix, box [box_rows x 64 cols], 128-byte swizzle, zero fill.
-bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {pitch_bytes};
-    const cuuint32_t box[2] = {BK, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline unsigned nblk(size_t total, int th) { return (unsigned)((total + th - 1) / th); }
@@ -340,14 +285,15 @@ struct TcState {
     int P2, P3;
     int splits, cps;            // FC split-K
     // packed weights
-    __half *w2p, *w3p, *wfcp;
-    float *w1f, *b1, *b2, *b3, *bfc, *whead, *bhead;
+    Conv1Plan pl1;
+    __half *w1p, *w2p, *w3p, *wfcp;
+    float *b1, *b2, *b3, *bfc, *whead, *bhead;
     unsigned* absmax;           // [L_COUNT]
     float *scale, *inv_scale;   // [L_COUNT] each
     // workspace
     __half *a1s, *a2, *a3;
     float *hpart, *h;
-    CUtensorMap mA2, mB2, mA3, mB3, mAfc, mBfc;
+    CUtensorMap mW1, mA2, mB2, mA3, mB3, mAfc, mBfc;
     int* status;
 };
 
@@ -357,6 +303,7 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     TcState* t = new (std::nothrow) TcState();
     if (!t) return HTS_ERR_ALLOC;
     t->g = g; t->max_batch = max_batch; t->status = status;
+    if (!conv1_plan(g, &t->pl1)) { delete t; return HTS_ERR_SHAPE; }
     t->H1s = (g.H1 + 1) / 2; t->W1s = (g.W1 + 1) / 2; t->P1s = t->H1s * t->W1s;
     t->P2 = g.H2 * g.W2; t->P3 = g.H3 * g.W3;
     const int chunks = g.F / BK;
@@ -366,7 +313,7 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     const size_t nb = (size_t)max_batch;
     auto A = [&](auto** p, size_t count) { return alloc(alloc_ctx, reinterpret_cast<void**>(p), count * sizeof(**p)); };
     bool ok = A(&t->w2p, (size_t)64 * 512) && A(&t->w3p, (size_t)64 * 576) && A(&t->wfcp, (size_t)512 * g.F) &&
-              A(&t->w1f, (size_t)32 * g.C * 64) && A(&t->b1, 32) && A(&t->b2, 64) && A(&t->b3, 64) && A(&t->bfc, 512) &&
+              A(&t->w1p, (size_t)32 * 4 * t->pl1.Cs) && A(&t->b1, 32) && A(&t->b2, 64) && A(&t->b3, 64) && A(&t->bfc, 512) &&
               A(&t->whead, (size_t)(g.A + 1) * 512) && A(&t->bhead, (size_t)g.A + 1) &&
               A(&t->absmax, L_COUNT) && A(&t->scale, L_COUNT) && A(&t->inv_scale, L_COUNT) &&
               A(&t->a1s, nb * t->P1s * 128) && A(&t->a2, nb * t->P2 * 64) && A(&t->a3, nb * g.F) &&
@@ -374,7 +321,8 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     if (!ok) { delete t; return HTS_ERR_ALLOC; }
     // cells of an odd-sized s2d border that conv1 never writes must hold finite numbers
     if (cudaMemset(t->a1s, 0, nb * t->P1s * 128 * 2) != cudaSuccess) { delete t; return cuda_fail(cudaGetLastError(), "cudaMemset"); }
-    ok = make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, BM) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
+    ok = make_map(&t->mW1, t->w1p, 32, 4 * t->pl1.Cs, (uint64_t)8 * t->pl1.Cs, 32) &&
+         make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, BM) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
          make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, BM) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
          make_map(&t->mAfc, t->a3, nb, g.F, (uint64_t)g.F * 2, BM) && make_map(&t->mBfc, t->wfcp, 512, g.F, (uint64_t)g.F * 2, 128);
     if (!ok) { delete t; return HTS_ERR_CUDA; }
@@ -398,11 +346,13 @@ hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s)
     }
     scales_kernel<<<1, 32, 0, s>>>(t->absmax, t->scale, t->inv_scale, 1.0f / 255.0f);
     HTS_LAUNCH_CHECK("scales");
+    hts_status st1 = conv1_pack_weights(t->pl1, bf(w.conv1_w), t->w1p, t->scale + L_CONV1, s);
+    if (st1 != HTS_OK) return st1;
     pack_conv2_kernel<<<nblk(64 * 512, 256), 256, 0, s>>>(bf(w.conv2_w), t->w2p, t->scale); HTS_LAUNCH_CHECK("pack_conv2");
     pack_conv3_kernel<<<nblk(64 * 576, 256), 256, 0, s>>>(bf(w.conv3_w), t->w3p, t->scale); HTS_LAUNCH_CHECK("pack_conv3");
     pack_fc_kernel<<<nblk((size_t)512 * g.F, 256), 256, 0, s>>>(bf(w.fc_w), t->wfcp, t->P3, t->scale); HTS_LAUNCH_CHECK("pack_fc");
     struct It { const void* p; float* q; size_t n; };
-    const It items[] = {{w.conv1_w, t->w1f, (size_t)32 * g.C * 64}, {w.conv1_b, t->b1, 32}, {w.conv2_b, t->b2, 64},
+    const It items[] = {{w.conv1_b, t->b1, 32}, {w.conv2_b, t->b2, 64},
                         {w.conv3_b, t->b3, 64}, {w.fc_b, t->bfc, 512}, {w.pi_w, t->whead, (size_t)g.A * 512},
                         {w.v_w, t->whead + (size_t)g.A * 512, 512}, {w.pi_b, t->bhead, (size_t)g.A}, {w.v_b, t->bhead + g.A, 1}};
     for (const It& it : items) {
@@ -416,9 +366,8 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cud
 {
     const Geometry& g = t->g;
     prof.begin(K_CONV1, s);
-    conv1_direct_s2d_kernel<<<nblk((size_t)n * 32 * g.H1 * g.W1, 256), 256, 0, s>>>(
-        obs, t->w1f, t->b1, t->a1s, n, g.C, g.H, g.W, g.H1, g.W1, t->P1s, t->W1s);
-    HTS_LAUNCH_CHECK("conv1_direct_s2d");
+    hts_status st = conv1_launch(t->pl1, t->mW1, obs, n, t->b1, t->inv_scale + L_CONV1, t->a1s, t->status, s);
+    if (st != HTS_OK) return st;
     prof.end(K_CONV1, s);
 
     GemmParams p{};
@@ -429,7 +378,7 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cud
     p.P_in = t->P1s; p.W_in = t->W1s; p.H_out = g.H2; p.W_out = g.W2; p.P_out = t->P2;
     p.bias = t->b2; p.out_h = t->a2; p.inv_scale = t->inv_scale + L_CONV2;
     prof.begin(K_CONV2, s);
-    hts_status st = launch_gemm<64, EPI_CONV>(t->mA2, t->mB2, p, dim3(nblk((size_t)n * t->P1s, BM), 1, 1), s);
+    st = launch_gemm<64, EPI_CONV>(t->mA2, t->mB2, p, dim3(nblk((size_t)n * t->P1s, BM), 1, 1), s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV2, s);
     // conv3: 3x3 taps on [H2, W2] x 64 -> [H3, W3] x 64
