@@ -1,0 +1,180 @@
+// conv2 / conv3 of the policy-value network as a persistent tcgen05 kernel.
+//
+// A stride-1 convolution on the flat pixel grid is a sum over filter taps of row-shifted GEMMs
+//     D[m, o] = sum_tap sum_c X[m + dy*W_in + dx, c] * W[o, tap, c].
+// Each CTA keeps the whole packed filter in shared memory and walks over 128-row tiles of the
+// activation matrix.  For a tile it loads rows [m0, m0 + 128 + largest shift) ONCE (one TMA box
+// per 64-channel plane, 128-byte swizzle) and every tap reads the same tile through a shared-
+// memory descriptor whose start address is moved by `shift` rows: the swizzle is a function of
+// the address bits, so a start that is a multiple of 128 bytes keeps the pattern intact.
+// Activation tiles and accumulators are double buffered: the copy of tile i+1 and the epilogue
+// of tile i-1 overlap the MMAs of tile i.  Rows whose pixel lies outside the output extent are
+// computed and dropped by the epilogue.
+#include "conv_res_tc.cuh"
+#include "tc_ptx.cuh"
+
+namespace hts {
+using namespace tc;
+
+namespace {
+
+constexpr int kThreads = 192;                   // warp 0 copies, warp 1 MMA issue, warps 2..5 epilogue
+constexpr int kChunkBytes = 64 * 128;           // one filter K chunk: 64 output channels x 128 bytes
+
+template <int TAPS, int CPT>
+__global__ void __launch_bounds__(kThreads)
+conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const ConvResParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t w_bar, a_full[2], a_empty[2], d_full[2], d_empty[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    volatile int* abortp = &abort_flag;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    constexpr int w_bytes = TAPS * CPT * kChunkBytes;
+    const int plane_bytes = p.tile_rows * 128;
+    const int a_bytes = CPT * plane_bytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles = (p.total_rows + 127) / 128;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&w_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&a_full[b], 1); mbar_init(&a_empty[b], 1);
+            mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 128);
+        }
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmW);
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&w_bar, w_bytes);
+            for (int g = 0; g < TAPS * CPT; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+            int it = 0;
+            for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
+                const int b = it & 1;
+                if (!mbar_wait(&a_empty[b], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 21)) break;
+                uint8_t* dst = sm + w_bytes + b * a_bytes;
+                mbar_arrive_expect_tx(&a_full[b], (uint32_t)a_bytes);
+                for (int pl = 0; pl < CPT; ++pl) tma_load_2d(dst + pl * plane_bytes, &tmA, pl * 64, tile * 128, &a_full[b]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_f16(0, 128, 64);
+            bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 22);
+            int it = 0;
+            for (int tile = blockIdx.x; alive && tile < tiles; tile += gridDim.x, ++it) {
+                const int b = it & 1;
+                const uint32_t ph = ((uint32_t)it >> 1) & 1u;
+                if (!mbar_wait(&a_full[b], ph, abortp, p.status, 23)) break;
+                if (!mbar_wait(&d_empty[b], ph ^ 1u, abortp, p.status, 24)) break;
+                tc_fence_after();
+                const uint32_t a_addr = base + w_bytes + b * a_bytes;
+                const uint32_t d_addr = tmem_d + b * 64;
+                uint32_t acc = 0;
+#pragma unroll
+                for (int tap = 0; tap < TAPS; ++tap) {
+#pragma unroll
+                    for (int pl = 0; pl < CPT; ++pl) {
+                        const uint64_t adesc = smem_desc_sw128(a_addr + pl * plane_bytes + p.tap_shift[tap] * 128);
+                        const uint64_t bdesc = smem_desc_sw128(base + (tap * CPT + pl) * kChunkBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) { mma_f16_ss(d_addr, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
+                    }
+                }
+                mma_commit(&a_empty[b]);
+                mma_commit(&d_full[b]);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int r = q * 32 + lane;
+        const float inv = *p.inv_scale;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
+            const int b = it & 1;
+            if (!mbar_wait(&d_full[b], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
+            tc_fence_after();
+            const long m = (long)tile * 128 + r;
+            const int env = (int)(m / p.P_in);
+            const int pix = (int)(m - (long)env * p.P_in);
+            const int y = pix / p.W_in, x = pix - y * p.W_in;
+            const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
+            __half* dst = p.out + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * 64;
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_d + b * 64 + ((uint32_t)(q * 32) << 16) + c, v);
+                tmem_ld_wait();
+                if (c == 32) {                           // accumulator fully read: hand it back
+                    tc_fence_before();
+                    mbar_arrive(&d_empty[b]);
+                }
+                if (valid) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            float a0 = fmaf(__uint_as_float(v[j + 2 * h]), inv, p.bias[c + j + 2 * h]);
+                            float a1 = fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, p.bias[c + j + 2 * h + 1]);
+                            a0 = fminf(fmaxf(a0, 0.f), 65504.f);
+                            a1 = fminf(fmaxf(a1, 0.f), 65504.f);
+                            __half2 t = __floats2half2_rn(a0, a1);
+                            pk[h] = *reinterpret_cast<uint32_t*>(&t);
+                        }
+                        *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            }
+        }
+    }
+    if (*abortp) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_d, 128);
+}
+
+}  // namespace
+
+template <int TAPS, int CPT>
+hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight_map, const ConvResParams& p,
+                           cudaStream_t s)
+{
+    static int sm_count = 0, smem_set = 0;
+    if (!sm_count) {
+        int dev = 0;
+        HTS_CUDA(cudaGetDevice(&dev));
+        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    const int smem = 1024 + TAPS * CPT * kChunkBytes + 2 * CPT * p.tile_rows * 128;
+    if (smem > 227 * 1024) return HTS_ERR_SHAPE;
+    if (smem > smem_set) {
+        HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        smem_set = smem;
+    }
+    const int tiles = (p.total_rows + 127) / 128;
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    conv_res_kernel<TAPS, CPT><<<grid, kThreads, smem, s>>>(act_map, weight_map, p);
+    HTS_LAUNCH_CHECK("conv_res_kernel");
+    return HTS_OK;
+}
+
+template hts_status conv_res_launch<4, 2>(const CUtensorMap&, const CUtensorMap&, const ConvResParams&, cudaStream_t);
+template hts_status conv_res_launch<9, 1>(const CUtensorMap&, const CUtensorMap&, const ConvResParams&, cudaStream_t);
+
+}  // namespace hts

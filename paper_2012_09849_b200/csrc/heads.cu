@@ -13,6 +13,7 @@ namespace {
 
 constexpr int kHidden = 512;
 constexpr int kMaxActions = 64;
+constexpr int kMaxSplits = 8;
 
 __device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1)
 {
@@ -66,31 +67,61 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
              float* __restrict__ values, float* __restrict__ entropy, float* __restrict__ logits_out,
              float* __restrict__ h_out)
 {
+    extern __shared__ float4 s_w4[];                   // [(A+1)*512] head weights, staged once per block
     __shared__ float s_out[8][kMaxActions + 1];
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int e = blockIdx.x * 8 + wib;
-    if (e >= n) return;
-
+    {
+        const float4* src = reinterpret_cast<const float4*>(whead);
+        const int total4 = (A + 1) * (kHidden / 4);
+        for (int i = threadIdx.x; i < total4; i += 256) s_w4[i] = src[i];
+    }
+    __syncthreads();
+    const float* sw = reinterpret_cast<const float*>(s_w4);
+    for (int e = blockIdx.x * 8 + wib; e < n; e += gridDim.x * 8) {
+    // hidden vector: split partials summed in index order (four splits' loads in flight at a time)
     float h[kHidden / 32];
 #pragma unroll
-    for (int i = 0; i < kHidden / 32; ++i) {
-        const int f = lane + 32 * i;
-        float v = h_partials[(size_t)e * kHidden + f];
-        if (fc_bias) {
-            for (int sp = 1; sp < num_splits; ++sp) v += h_partials[sp * split_stride + (size_t)e * kHidden + f];
-            v += fc_bias[f];
-            v = v > 0.f ? v : 0.f;
-        }
-        h[i] = v;
-        if (h_out) h_out[(size_t)e * kHidden + f] = v;
-    }
-    for (int o = 0; o <= A; ++o) {
-        const float* wr = whead + (size_t)o * kHidden;
-        float acc = 0.f;
+    for (int i = 0; i < kHidden / 32; ++i) h[i] = 0.f;
 #pragma unroll
-        for (int i = 0; i < kHidden / 32; ++i) acc = fmaf(wr[lane + 32 * i], h[i], acc);
-        acc = warp_sum(acc);
-        if (lane == 0) s_out[wib][o] = acc + bhead[o];
+    for (int sp0 = 0; sp0 < kMaxSplits; sp0 += 4) {
+        if (sp0 < num_splits) {
+            float part[4][kHidden / 32];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int i = 0; i < kHidden / 32; ++i)
+                    part[j][i] = (sp0 + j < num_splits)
+                                     ? h_partials[(sp0 + j) * split_stride + (size_t)e * kHidden + lane + 32 * i] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int i = 0; i < kHidden / 32; ++i)
+                    if (sp0 + j < num_splits) h[i] = (sp0 + j == 0) ? part[j][i] : h[i] + part[j][i];
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kHidden / 32; ++i) {
+        float v = h[i];
+        if (fc_bias) { v += fc_bias[lane + 32 * i]; v = v > 0.f ? v : 0.f; }
+        h[i] = v;
+        if (h_out) h_out[(size_t)e * kHidden + lane + 32 * i] = v;
+    }
+    for (int o0 = 0; o0 <= A; o0 += 4) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int o = (o0 + j <= A) ? o0 + j : A;
+#pragma unroll
+            for (int i = 0; i < kHidden / 32; ++i) acc[j] = fmaf(sw[o * kHidden + lane + 32 * i], h[i], acc[j]);
+        }
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], m);
+        if (lane < 4 && o0 + lane <= A) {
+            const float mine = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
+            s_out[wib][o0 + lane] = mine + bhead[o0 + lane];
+        }
     }
     __syncwarp();
     const float* lg = s_out[wib];
@@ -128,6 +159,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
         values[e] = lg[A];
         entropy[e] = ent;
     }
+    __syncwarp();                                      // s_out[wib] is reused by the next environment
+    }
 }
 
 }  // namespace
@@ -138,7 +171,22 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
                         uint64_t seed, int n, int32_t* actions, float* logp, float* values,
                         float* entropy, float* logits, float* h_out, cudaStream_t s)
 {
-    heads_kernel<<<(n + 7) / 8, 256, 0, s>>>(h_partials, num_splits, split_stride, fc_bias, whead, bhead, A,
+    if (num_splits < 1 || num_splits > kMaxSplits) return HTS_ERR_INVALID_ARG;
+    const size_t smem = (size_t)(A + 1) * kHidden * sizeof(float);
+    static size_t smem_set = 48 * 1024;
+    if (smem > smem_set) {
+        HTS_CUDA(cudaFuncSetAttribute(heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        smem_set = smem;
+    }
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        HTS_CUDA(cudaGetDevice(&dev));
+        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    int blocks = (n + 7) / 8;
+    if (blocks > 2 * sm_count) blocks = 2 * sm_count;
+    heads_kernel<<<blocks, 256, smem, s>>>(h_partials, num_splits, split_stride, fc_bias, whead, bhead, A,
                                            env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu),
                                            (uint32_t)(seed >> 32), n, actions, logp, values, entropy,
                                            logits, h_out);

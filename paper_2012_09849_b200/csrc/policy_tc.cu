@@ -24,6 +24,7 @@
 #include "tc_ptx.cuh"
 #include "tc_host.cuh"
 #include "conv1_tc.cuh"
+#include "conv_res_tc.cuh"
 
 namespace hts {
 using namespace tc;
@@ -294,6 +295,7 @@ struct TcState {
     __half *a1s, *a2, *a3;
     float *hpart, *h;
     CUtensorMap mW1, mA2, mB2, mA3, mB3, mAfc, mBfc;
+    int rows2, rows3;           // activation tile rows of conv2 / conv3
     int* status;
 };
 
@@ -321,9 +323,12 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     if (!ok) { delete t; return HTS_ERR_ALLOC; }
     // cells of an odd-sized s2d border that conv1 never writes must hold finite numbers
     if (cudaMemset(t->a1s, 0, nb * t->P1s * 128 * 2) != cudaSuccess) { delete t; return cuda_fail(cudaGetLastError(), "cudaMemset"); }
+    t->rows2 = conv_res_tile_rows(t->W1s + 1);
+    t->rows3 = conv_res_tile_rows(2 * g.W2 + 2);
+    if (t->rows2 > 256 || t->rows3 > 256) { delete t; return HTS_ERR_SHAPE; }
     ok = make_map(&t->mW1, t->w1p, 32, 4 * t->pl1.Cs, (uint64_t)8 * t->pl1.Cs, 32) &&
-         make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, BM) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
-         make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, BM) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
+         make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, t->rows2) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
+         make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, t->rows3) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
          make_map(&t->mAfc, t->a3, nb, g.F, (uint64_t)g.F * 2, BM) && make_map(&t->mBfc, t->wfcp, 512, g.F, (uint64_t)g.F * 2, 128);
     if (!ok) { delete t; return HTS_ERR_CUDA; }
     *out = t;
@@ -370,26 +375,28 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cud
     if (st != HTS_OK) return st;
     prof.end(K_CONV1, s);
 
-    GemmParams p{};
-    p.status = t->status; p.n_env = n;
     // conv2: 2x2 taps on the s2d grid [H1s, W1s] with 128 channels -> [H2, W2] x 64
-    p.taps = 4; p.cpt = 2; p.nk = 8;
-    p.tap_shift[0] = 0; p.tap_shift[1] = 1; p.tap_shift[2] = t->W1s; p.tap_shift[3] = t->W1s + 1;
-    p.P_in = t->P1s; p.W_in = t->W1s; p.H_out = g.H2; p.W_out = g.W2; p.P_out = t->P2;
-    p.bias = t->b2; p.out_h = t->a2; p.inv_scale = t->inv_scale + L_CONV2;
+    ConvResParams c{};
+    c.status = t->status; c.n_env = n;
+    c.tap_shift[0] = 0; c.tap_shift[1] = 1; c.tap_shift[2] = t->W1s; c.tap_shift[3] = t->W1s + 1;
+    c.tile_rows = t->rows2; c.total_rows = n * t->P1s;
+    c.P_in = t->P1s; c.W_in = t->W1s; c.H_out = g.H2; c.W_out = g.W2; c.P_out = t->P2;
+    c.bias = t->b2; c.out = t->a2; c.inv_scale = t->inv_scale + L_CONV2;
     prof.begin(K_CONV2, s);
-    st = launch_gemm<64, EPI_CONV>(t->mA2, t->mB2, p, dim3(nblk((size_t)n * t->P1s, BM), 1, 1), s);
+    st = conv_res_launch<4, 2>(t->mA2, t->mB2, c, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV2, s);
     // conv3: 3x3 taps on [H2, W2] x 64 -> [H3, W3] x 64
-    p.taps = 9; p.cpt = 1; p.nk = 9;
-    for (int dy = 0; dy < 3; ++dy) for (int dx = 0; dx < 3; ++dx) p.tap_shift[dy * 3 + dx] = dy * g.W2 + dx;
-    p.P_in = t->P2; p.W_in = g.W2; p.H_out = g.H3; p.W_out = g.W3; p.P_out = t->P3;
-    p.bias = t->b3; p.out_h = t->a3; p.inv_scale = t->inv_scale + L_CONV3;
+    for (int dy = 0; dy < 3; ++dy) for (int dx = 0; dx < 3; ++dx) c.tap_shift[dy * 3 + dx] = dy * g.W2 + dx;
+    c.tile_rows = t->rows3; c.total_rows = n * t->P2;
+    c.P_in = t->P2; c.W_in = g.W2; c.H_out = g.H3; c.W_out = g.W3; c.P_out = t->P3;
+    c.bias = t->b3; c.out = t->a3; c.inv_scale = t->inv_scale + L_CONV3;
     prof.begin(K_CONV3, s);
-    st = launch_gemm<64, EPI_CONV>(t->mA3, t->mB3, p, dim3(nblk((size_t)n * t->P2, BM), 1, 1), s);
+    st = conv_res_launch<9, 1>(t->mA3, t->mB3, c, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV3, s);
+    GemmParams p{};
+    p.status = t->status; p.n_env = n;
     // FC: [n, F] x [512, F]^T, K split across blockIdx.z
     p.taps = 1; p.cpt = g.F / BK; p.nk = t->cps; p.tap_shift[0] = 0;
     p.out_f32 = t->hpart; p.split_stride = (size_t)t->max_batch * 512; p.ldo = 512; p.inv_scale = t->inv_scale + L_FC;
