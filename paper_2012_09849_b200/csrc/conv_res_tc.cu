@@ -7,8 +7,8 @@
 // per 64-channel plane, 128-byte swizzle) and every tap reads the same tile through a shared-
 // memory descriptor whose start address is moved by `shift` rows: the swizzle is a function of
 // the address bits, so a start that is a multiple of 128 bytes keeps the pattern intact.
-// Activation tiles and accumulators are double buffered: the copy of tile i+1 and the epilogue
-// of tile i-1 overlap the MMAs of tile i.  Rows whose pixel lies outside the output extent are
+// Activation tiles sit in a 3- or 4-deep ring and the accumulator is double buffered, each
+// buffer with its own four epilogue warps: copies, MMAs and epilogues of different tiles overlap.  Rows whose pixel lies outside the output extent are
 // computed and dropped by the epilogue.
 #include "conv_res_tc.cuh"
 #include "tc_ptx.cuh"
@@ -18,15 +18,23 @@ using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 192;                   // warp 0 copies, warp 1 MMA issue, warps 2..5 epilogue
+constexpr int kThreads = 320;                   // warp 0 copies, warp 1 MMA issue, warps 2..5 and 6..9 epilogue
 constexpr int kChunkBytes = 64 * 128;           // one filter K chunk: 64 output channels x 128 bytes
 
-template <int TAPS, int CPT>
+// 256-bit store of eight packed half2 (one 32-byte sector)
+__device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&v)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
+template <int TAPS, int CPT, int NST>
 __global__ void __launch_bounds__(kThreads)
 conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const ConvResParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, a_full[2], a_empty[2], d_full[2], d_empty[2];
+    __shared__ uint64_t w_bar, a_full[NST], a_empty[NST], d_full[2], d_empty[2];
+    __shared__ float s_bias[64];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     volatile int* abortp = &abort_flag;
@@ -41,15 +49,14 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&a_full[b], 1); mbar_init(&a_empty[b], 1);
-            mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 128);
-        }
+        for (int b = 0; b < NST; ++b) { mbar_init(&a_full[b], 1); mbar_init(&a_empty[b], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 128); }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmW);
     }
+    if (threadIdx.x >= 64 && threadIdx.x < 128) s_bias[threadIdx.x - 64] = p.bias[threadIdx.x - 64];
     if (warp == 1) tmem_alloc(&tmem_slot, 128);
     tc_fence_before();
     __syncthreads();
@@ -62,8 +69,8 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int g = 0; g < TAPS * CPT; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
             int it = 0;
             for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
-                const int b = it & 1;
-                if (!mbar_wait(&a_empty[b], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 21)) break;
+                const int b = it % NST;
+                if (!mbar_wait(&a_empty[b], (((uint32_t)(it / NST)) & 1u) ^ 1u, abortp, p.status, 21)) break;
                 uint8_t* dst = sm + w_bytes + b * a_bytes;
                 mbar_arrive_expect_tx(&a_full[b], (uint32_t)a_bytes);
                 for (int pl = 0; pl < CPT; ++pl) tma_load_2d(dst + pl * plane_bytes, &tmA, pl * 64, tile * 128, &a_full[b]);
@@ -75,13 +82,12 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 22);
             int it = 0;
             for (int tile = blockIdx.x; alive && tile < tiles; tile += gridDim.x, ++it) {
-                const int b = it & 1;
-                const uint32_t ph = ((uint32_t)it >> 1) & 1u;
-                if (!mbar_wait(&a_full[b], ph, abortp, p.status, 23)) break;
-                if (!mbar_wait(&d_empty[b], ph ^ 1u, abortp, p.status, 24)) break;
+                const int b = it % NST, db = it & 1;
+                if (!mbar_wait(&a_full[b], ((uint32_t)(it / NST)) & 1u, abortp, p.status, 23)) break;
+                if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 24)) break;
                 tc_fence_after();
                 const uint32_t a_addr = base + w_bytes + b * a_bytes;
-                const uint32_t d_addr = tmem_d + b * 64;
+                const uint32_t d_addr = tmem_d + db * 64;
                 uint32_t acc = 0;
 #pragma unroll
                 for (int tap = 0; tap < TAPS; ++tap) {
@@ -94,17 +100,18 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                 }
                 mma_commit(&a_empty[b]);
-                mma_commit(&d_full[b]);
+                mma_commit(&d_full[db]);
             }
         }
     } else {
-        const int q = warp & 3;
+        // two groups of four warps; group g owns accumulator buffer g, i.e. every other tile
+        const int grp = (warp - 2) >> 2;
+        const int q = warp & 3;                         // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;
         const float inv = *p.inv_scale;
-        int it = 0;
-        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
-            const int b = it & 1;
-            if (!mbar_wait(&d_full[b], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
+        int it = grp;
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < tiles; tile += 2 * gridDim.x, it += 2) {
+            if (!mbar_wait(&d_full[grp], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
             tc_fence_after();
             const long m = (long)tile * 128 + r;
             const int env = (int)(m / p.P_in);
@@ -112,29 +119,30 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int y = pix / p.W_in, x = pix - y * p.W_in;
             const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
             __half* dst = p.out + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * 64;
+            uint32_t v0[32], v1[32];
+            const uint32_t taddr = tmem_d + grp * 64 + ((uint32_t)(q * 32) << 16);
+            tmem_ld_32x32(taddr, v0);
+            tmem_ld_32x32(taddr + 32, v1);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(&d_empty[grp]);                 // accumulator is in registers: hand it back
+            if (valid) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_d + b * 64 + ((uint32_t)(q * 32) << 16) + c, v);
-                tmem_ld_wait();
-                if (c == 32) {                           // accumulator fully read: hand it back
-                    tc_fence_before();
-                    mbar_arrive(&d_empty[b]);
-                }
-                if (valid) {
+                for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        uint32_t pk[4];
+                    for (int j = 0; j < 32; j += 16) {
+                        uint32_t pk[8];
 #pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            float a0 = fmaf(__uint_as_float(v[j + 2 * h]), inv, p.bias[c + j + 2 * h]);
-                            float a1 = fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, p.bias[c + j + 2 * h + 1]);
-                            a0 = fminf(fmaxf(a0, 0.f), 65504.f);
-                            a1 = fminf(fmaxf(a1, 0.f), 65504.f);
-                            __half2 t = __floats2half2_rn(a0, a1);
+                        for (int h = 0; h < 8; ++h) {
+                            const int c = j + 2 * h;
+                            const float x0 = __uint_as_float(half ? v1[c] : v0[c]);
+                            const float x1 = __uint_as_float(half ? v1[c + 1] : v0[c + 1]);
+                            __half2 t = __floats2half2_rn(fmaf(x0, inv, s_bias[half * 32 + c]),
+                                                          fmaf(x1, inv, s_bias[half * 32 + c + 1]));
+                            t = __hmin2(__hmax2(t, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
                             pk[h] = *reinterpret_cast<uint32_t*>(&t);
                         }
-                        *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        st_global_v8(dst + half * 32 + j, pk);
                     }
                 }
             }
@@ -161,15 +169,16 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
         HTS_CUDA(cudaGetDevice(&dev));
         HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
-    const int smem = 1024 + TAPS * CPT * kChunkBytes + 2 * CPT * p.tile_rows * 128;
+    constexpr int NST = CPT == 2 ? 3 : 4;        // activation tiles in flight
+    const int smem = 1024 + TAPS * CPT * kChunkBytes + NST * CPT * p.tile_rows * 128;
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;
     if (smem > smem_set) {
-        HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         smem_set = smem;
     }
     const int tiles = (p.total_rows + 127) / 128;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    conv_res_kernel<TAPS, CPT><<<grid, kThreads, smem, s>>>(act_map, weight_map, p);
+    conv_res_kernel<TAPS, CPT, NST><<<grid, kThreads, smem, s>>>(act_map, weight_map, p);
     HTS_LAUNCH_CHECK("conv_res_kernel");
     return HTS_OK;
 }
