@@ -56,6 +56,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     __shared__ uint64_t w_bar, u8_full[2], u8_empty[2], a_ready, d_full;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float s_bias[32];
     volatile int* abortp = &abort_flag;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -81,6 +82,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         fence_barrier_init();
         tma_prefetch_desc(&tmW);
     }
+    if (threadIdx.x >= 32 && threadIdx.x < 64) s_bias[threadIdx.x - 32] = p.bias[threadIdx.x - 32];
     if (warp == 0) tmem_alloc(&tmem_slot, 32);
     tc_fence_before();
     __syncthreads();
@@ -139,64 +141,65 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         const int q = warp & 3;                          // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;                   // tile row handled in the epilogue
         const float inv = *p.inv_scale;
-        float bias[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) bias[j] = p.bias[j];
+        // convert: thread owns one 16-byte chunk position qq of every 16th pixel
+        const int qq = tid & 7, slot = tid >> 3;
+        const int src_q = ((qq >> 1) * band_in_rows + 2 * (qq & 1)) * pl.W;     // channel (qq>>1) of a plane, row pair (qq&1)
+        const int plane_src = 4 * band_in_rows * pl.W;                          // four channels per plane
+        const int ey = row / pl.Ws, ex = row - ey * pl.Ws;                       // epilogue pixel of this thread
         int it = 0;
         for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
             const int s = it & 1;
             const int env = u / pl.bands, band = u - env * pl.bands;
             const int y0 = band * pl.R;
             int in_rows = pl.H - 4 * y0; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
-            const int s2d_rows = in_rows >> 2;           // space-to-depth rows present in this band
-            if (!mbar_wait(&u8_full[s], ((uint32_t)it >> 1) & 1u, abortp, p.status, 14)) break;
-            // ---- convert: item = (plane, pixel, 16-byte chunk): 2 rows x 4 bytes of one channel
-            const uint8_t* src = s_u8 + s * pl.u8_stage_bytes;
-            const int pixels = s2d_rows * pl.Ws;
-            const int items = pl.cpt * pixels * 8;
-            for (int i = tid; i < items; i += kWorkers) {
-                const int qq = i & 7;
-                const int rest = i >> 3;
-                const int pln = rest / pixels;
-                const int ps = rest - pln * pixels;
-                const int ys = ps / pl.Ws, xs = ps - ys * pl.Ws;
-                const int c = pln * 4 + (qq >> 1);
-                const uint8_t* s0 = src + (c * band_in_rows + 4 * ys + 2 * (qq & 1)) * pl.W + 4 * xs;
-                const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
-                const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
-                uint4 o;
-                u8x4_to_h4(w0, o.x, o.y);
-                u8x4_to_h4(w1, o.z, o.w);
-                *reinterpret_cast<uint4*>(s_tile + pln * plane_bytes + ps * 128 + ((qq ^ (ps & 7)) << 4)) = o;
+            const int pixels = (in_rows >> 2) * pl.Ws;   // space-to-depth pixels present in this band
+            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)it >> 1) & 1u, abortp, p.status, 14)) break;
+            const uint8_t* src = s_u8 + s * pl.u8_stage_bytes + src_q;
+            for (int pln = 0; pln < pl.cpt; ++pln) {
+                uint8_t* dplane = s_tile + pln * plane_bytes;
+                const uint8_t* splane = src + pln * plane_src;
+                int ys = 0, xs = slot;
+                while (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
+                for (int ps = slot; ps < pixels; ps += 16) {
+                    const uint8_t* s0 = splane + (4 * ys) * pl.W + 4 * xs;
+                    const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
+                    const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
+                    uint4 o;
+                    u8x4_to_h4(w0, o.x, o.y);
+                    u8x4_to_h4(w1, o.z, o.w);
+                    *reinterpret_cast<uint4*>(dplane + ps * 128 + ((qq ^ (ps & 7)) << 4)) = o;
+                    xs += 16;
+                    while (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
+                }
             }
             fence_async_proxy();                         // tile stores -> visible to the tensor core's reads
             mbar_arrive(&u8_empty[s]);
             mbar_arrive(&a_ready);
             // ---- epilogue
-            if (!mbar_wait(&d_full, (uint32_t)it & 1u, abortp, p.status, 15)) break;
+            if (!mbar_wait_warp(&d_full, (uint32_t)it & 1u, abortp, p.status, 15)) break;
             tc_fence_after();
             uint32_t v[32];
             tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16), v);
             tmem_ld_wait();
             tc_fence_before();
-            const int y = row / pl.Ws, x = row - y * pl.Ws;
-            const int yy = y0 + y;
-            if (y < pl.R && yy < pl.H1 && x < pl.W1) {
-                __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (x >> 1)) * 128 +
-                              ((yy & 1) * 2 + (x & 1)) * 32;
+            const int yy = y0 + ey;
+            if (ey < pl.R && yy < pl.H1 && ex < pl.W1) {
+                __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (ex >> 1)) * 128 +
+                              ((yy & 1) * 2 + (ex & 1)) * 32;
 #pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    uint32_t pk[4];
+                for (int j = 0; j < 32; j += 16) {
+                    uint32_t pk[8];
 #pragma unroll
-                    for (int h = 0; h < 4; ++h) {
-                        float a = fmaf(__uint_as_float(v[j + 2 * h]), inv, bias[j + 2 * h]);
-                        float b = fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, bias[j + 2 * h + 1]);
-                        a = fminf(fmaxf(a, 0.f), 65504.f);
-                        b = fminf(fmaxf(b, 0.f), 65504.f);
-                        __half2 t = __floats2half2_rn(a, b);
+                    for (int h = 0; h < 8; ++h) {
+                        const int c = j + 2 * h;
+                        __half2 t = __floats2half2_rn(fmaf(__uint_as_float(v[c]), inv, s_bias[c]),
+                                                      fmaf(__uint_as_float(v[c + 1]), inv, s_bias[c + 1]));
+                        t = __hmin2(__hmax2(t, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
                         pk[h] = *reinterpret_cast<uint32_t*>(&t);
                     }
-                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                   "r"(pk[6]), "r"(pk[7]) : "memory");
                 }
             }
         }
@@ -262,6 +265,9 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
     }
     if (max_smem_set < pl.smem_bytes) {
         HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
+        // every kernel of the step asks for the largest shared-memory carve-out, so that the SMs are not
+        // re-partitioned between consecutive kernels
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         max_smem_set = pl.smem_bytes;
     }
     const int per_sm = (227 * 1024) / (pl.smem_bytes + 1024) > 4 ? 4 : (227 * 1024) / (pl.smem_bytes + 1024);

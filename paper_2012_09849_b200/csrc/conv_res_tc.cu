@@ -111,7 +111,7 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const float inv = *p.inv_scale;
         int it = grp;
         for (int tile = blockIdx.x + grp * gridDim.x; tile < tiles; tile += 2 * gridDim.x, it += 2) {
-            if (!mbar_wait(&d_full[grp], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
+            if (!mbar_wait_warp(&d_full[grp], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
             tc_fence_after();
             const long m = (long)tile * 128 + r;
             const int env = (int)(m / p.P_in);
@@ -174,6 +174,7 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;
     if (smem > smem_set) {
         HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         smem_set = smem;
     }
     const int tiles = (p.total_rows + 127) / 128;

@@ -174,6 +174,11 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
     if (num_splits < 1 || num_splits > kMaxSplits) return HTS_ERR_INVALID_ARG;
     const size_t smem = (size_t)(A + 1) * kHidden * sizeof(float);
     static size_t smem_set = 48 * 1024;
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        HTS_CUDA(cudaFuncSetAttribute(heads_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        carveout_set = true;
+    }
     if (smem > smem_set) {
         HTS_CUDA(cudaFuncSetAttribute(heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         smem_set = smem;

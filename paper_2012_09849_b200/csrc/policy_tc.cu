@@ -129,7 +129,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // epilogue warps 2..5: warp w may touch TMEM lanes [32*(w%4), 32*(w%4)+32)
         const int q = warp & 3;
         const int r = q * 32 + lane;                    // row of the tile = TMEM lane
-        const bool ok = mbar_wait(&accum_bar, 0, abortp, p.status, 3);
+        const bool ok = mbar_wait_warp(&accum_bar, 0, abortp, p.status, 3);
         tc_fence_after();
         if (ok) {
             const long m = (long)m0 + r;
@@ -270,6 +270,7 @@ hts_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPar
     static bool attr_set = false;
     if (!attr_set) {
         HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         attr_set = true;
     }
     gemm_tc_kernel<BN, EPI><<<grid, 192, smem, s>>>(a, b, p);

@@ -37,21 +37,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 // Bounded wait.  Gives up after ~2e9 clock ticks (about a second) or as soon as another thread
 // of the block has given up (*abort_flag != 0); then records `code` in the device status word
 // and returns false.  Callers leave their loops, the block drains and returns normally.
+// Failed polls back off with a short sleep: polling threads read shared memory, and the tensor
+// core fetches its operands from the same shared memory.
 constexpr long long kWaitLimitTicks = 2000000000LL;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitTicks) {
-            *abort_flag = 1;
-            if (status) atomicCAS(status, 0, code);
-            return false;
+    for (int spins = 0;; ++spins) {
+        __nanosleep(32);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 63) == 63) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitTicks) {
+                *abort_flag = 1;
+                if (status) atomicCAS(status, 0, code);
+                return false;
+            }
         }
     }
+}
+// The same for a whole warp (all 32 lanes must call it together): lane 0 polls, the others
+// join once the phase has completed, so a waiting warp costs one poller instead of 32.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code)
+{
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, code);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) {
+        while (!mbar_try_wait(bar, parity)) { }         // completes at once: the phase is already over
+    }
+    return ok;
 }
 
 // ---- TMA (tiled, 2-D, shared::cta destination of this CTA, completion on an mbarrier) ---------
