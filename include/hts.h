@@ -167,6 +167,39 @@ hts_status hts_gae_host(const float *rewards, const float *values, const uint8_t
                         const float *bootstrap, float gamma, float lambda, int32_t T,
                         int32_t N, float *advantages, float *returns, void *cuda_stream);
 
+/* The actor step for callers that must not allocate.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, for example an
+ * inference loop inside a process whose device memory is fully handed to another
+ * allocator or pool, a plug-in that may not change the host's memory footprint, or a
+ * latency-critical loop that cannot afford the implicit device synchronisation of an
+ * allocation.  hts_policy_create allocates its workspace with cudaMalloc; this call
+ * needs no context and allocates nothing, neither itself nor through a library.
+ *
+ * What it does: the fp32 check-path arithmetic of hts_policy_step (same kernels, same
+ * results bit for bit) on the caller's own fp32 weights, read in place from `w`
+ * (PyTorch layouts, DEVICE pointers; desc->weight_dtype must be HTS_DTYPE_FP32,
+ * desc->max_batch is ignored).  Inputs and outputs as for hts_policy_step.
+ *
+ * Scratch: hidden activations and the stacked head weights go to a fixed array of
+ * 2^20 floats (4 MiB) that is part of the library image; every GPU that loads the
+ * library holds it until the process exits.  A call whose
+ *   n*(32*H1*W1 + 64*H2*W2 + 64*H3*W3 + 512) + (A+1)*513
+ * floats do not fit (more than 48 observations of 4x84x84 with 18 actions) is refused
+ * with HTS_ERR_INVALID_ARG.  The array is shared by all calls and keeps the previous
+ * call's contents; the call overwrites every part it reads, so nothing needs clearing,
+ * but two calls whose GPU work overlaps (different streams, or threads) race on it:
+ * serialise them.  The first call on each device looks up the array's device address
+ * (with that device current); make that first call before starting any stream capture.
+ * Errors: INVALID_ARG (NULL, n < 1, too large for the scratch), SHAPE, UNSUPPORTED
+ * (weights not fp32, device index above 63), CUDA.                                   */
+hts_status hts_policy_step_noalloc(const hts_net_desc *desc, const hts_weights *w, const uint8_t *obs,
+                                   const int32_t *env_ids, const int32_t *t_per_env, int32_t t,
+                                   uint64_t seed, int32_t n, int32_t *actions, float *logp,
+                                   float *values, float *entropy, float *logits_or_null,
+                                   void *cuda_stream);
+
 /* Number of kernel launches this library has enqueued since it was loaded
  * (all contexts, all streams); for launch accounting by a benchmark.              */
 uint64_t hts_launch_count(void);

@@ -25,7 +25,7 @@ WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b"
 EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_host",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
-           "hts_gae_host", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
+           "hts_gae_host", "hts_policy_step_noalloc", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
 
 
 class HtsError(RuntimeError):
@@ -80,6 +80,8 @@ def lib():
         gae = [vp, vp, vp, vp, f32, f32, i32, i32, vp, vp, vp]
         L.hts_gae.argtypes = gae
         L.hts_gae_host.argtypes = gae
+        L.hts_policy_step_noalloc.argtypes = [C.POINTER(hts_net_desc), C.POINTER(hts_weights)] + step[1:]
+        L.hts_policy_step_noalloc.restype = C.c_int
         L.hts_launch_count.restype = C.c_uint64
         L.hts_last_cuda_error.restype = C.c_char_p
         L.hts_status_string.restype = C.c_char_p
@@ -186,6 +188,17 @@ def hts_gae(rewards, values, dones, bootstrap, gamma, lam, T, N, advantages, ret
 def hts_gae_host(rewards, values, dones, bootstrap, gamma, lam, T, N, advantages, returns, stream=None) -> None:
     _check(lib().hts_gae_host(_ptr(rewards), _ptr(values), _ptr(dones), _ptr(bootstrap), float(gamma), float(lam),
                               int(T), int(N), _ptr(advantages), _ptr(returns), _stream(stream)), "hts_gae_host")
+
+
+def hts_policy_step_noalloc(C_, H, W, num_actions, weights: dict, obs, env_ids, t_per_env, t, seed, n,
+                            actions, logp, values, entropy, logits=None, stream=None) -> None:
+    """Actor step without any allocation: fp32 weights (dict of CUDA float32 tensors) are read in place and
+    the hidden activations use the library's fixed 4 MiB scratch array (see hts.h for the limits)."""
+    d = hts_net_desc(C_, H, W, num_actions, HTS_DTYPE_FP32, n)
+    w = hts_weights(**{k: _ptr(weights[k]) for k in WEIGHT_NAMES})
+    _check(lib().hts_policy_step_noalloc(C.byref(d), C.byref(w), _ptr(obs), _ptr(env_ids), _ptr(t_per_env), int(t),
+                                         int(seed), int(n), _ptr(actions), _ptr(logp), _ptr(values), _ptr(entropy),
+                                         _ptr(logits), _stream(stream)), "hts_policy_step_noalloc")
 
 
 def hts_launch_count() -> int:

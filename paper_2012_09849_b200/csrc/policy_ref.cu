@@ -109,3 +109,69 @@ hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspac
 }
 
 }  // namespace hts
+
+// ---- actor step that allocates nothing ----------------------------------------------------------
+// Scratch for hts_policy_step_noalloc: hidden activations of the four layers plus the stacked
+// head weights, as floats.  It lives in the library image, so every GPU that loads the library
+// carries these 4 MiB until the process exits.
+namespace {
+constexpr size_t kNoAllocFloats = size_t(1) << 20;
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocFloats];
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices] = {};       // device address of the array, looked up once per device
+}  // namespace
+
+extern "C" hts_status hts_policy_step_noalloc(const hts_net_desc* d, const hts_weights* w, const uint8_t* obs,
+                                              const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
+                                              uint64_t seed, int32_t n, int32_t* actions, float* logp,
+                                              float* values, float* entropy, float* logits_or_null,
+                                              void* cuda_stream)
+{
+    using namespace hts;
+    if (!d || !w || !obs || !env_ids || !actions || !logp || !values || !entropy) return HTS_ERR_INVALID_ARG;
+    const void* const* wp = reinterpret_cast<const void* const*>(w);
+    for (int i = 0; i < 12; ++i) if (!wp[i]) return HTS_ERR_INVALID_ARG;
+    if (d->weight_dtype != HTS_DTYPE_FP32) return HTS_ERR_UNSUPPORTED;
+    if (n < 1 || d->C < 1 || d->num_actions < 1 || d->num_actions > 64) return HTS_ERR_INVALID_ARG;
+    if (d->H % 4 || d->W % 4 || d->H < 8 || d->W < 8) return HTS_ERR_SHAPE;
+    Geometry g{};
+    g.C = d->C; g.H = d->H; g.W = d->W; g.A = d->num_actions;
+    g.H1 = conv_out(g.H, 8, 4); g.W1 = conv_out(g.W, 8, 4);
+    if (g.H1 < 4 || g.W1 < 4) return HTS_ERR_SHAPE;
+    g.H2 = conv_out(g.H1, 4, 2); g.W2 = conv_out(g.W1, 4, 2);
+    if (g.H2 < 3 || g.W2 < 3) return HTS_ERR_SHAPE;
+    g.H3 = conv_out(g.H2, 3, 1); g.W3 = conv_out(g.W2, 3, 1);
+    g.F = 64 * g.H3 * g.W3;
+    const size_t nn = (size_t)n;
+    const size_t f_a1 = nn * 32 * g.H1 * g.W1, f_a2 = nn * 64 * g.H2 * g.W2, f_a3 = nn * g.F, f_h = nn * 512;
+    const size_t f_wh = (size_t)(g.A + 1) * 512, f_bh = (size_t)g.A + 1;
+    if (f_a1 + f_a2 + f_a3 + f_h + f_wh + f_bh > kNoAllocFloats) return HTS_ERR_INVALID_ARG;   // batch too large for the fixed scratch
+
+    int dev = 0;
+    HTS_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return HTS_ERR_UNSUPPORTED;
+    if (!g_noalloc_ptr[dev]) {
+        // In host code the array's name is only a handle: the kernels need its device address.
+        float* ptr = nullptr;
+        HTS_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch));
+        g_noalloc_ptr[dev] = ptr;
+    }
+    float* base = g_noalloc_ptr[dev];
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    RefWorkspace ws{base, base + f_a1, base + f_a1 + f_a2, base + f_a1 + f_a2 + f_a3};
+    float* whead = ws.h + f_h;
+    float* bhead = whead + f_wh;
+    // every scratch float is written before it is read, so nothing has to start at zero
+    HTS_CUDA(cudaMemcpyAsync(whead, w->pi_w, (size_t)g.A * 512 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    HTS_CUDA(cudaMemcpyAsync(whead + (size_t)g.A * 512, w->v_w, 512 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    HTS_CUDA(cudaMemcpyAsync(bhead, w->pi_b, (size_t)g.A * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    HTS_CUDA(cudaMemcpyAsync(bhead + g.A, w->v_b, sizeof(float), cudaMemcpyDeviceToDevice, s));
+    auto f = [](const void* p) { return const_cast<float*>(static_cast<const float*>(p)); };
+    const RefWeights rw{f(w->conv1_w), f(w->conv1_b), f(w->conv2_w), f(w->conv2_b), f(w->conv3_w), f(w->conv3_b),
+                        f(w->fc_w), f(w->fc_b), whead, bhead};
+    Profiler off;
+    hts_status st = ref_forward(g, rw, ws, obs, n, off, s);
+    if (st != HTS_OK) return st;
+    return launch_heads(ws.h, 1, 0, nullptr, whead, bhead, g.A, env_ids, t_per_env, t, seed, n, actions, logp,
+                        values, entropy, logits_or_null, nullptr, s);
+}
