@@ -22,6 +22,26 @@ hts_status cuda_fail(cudaError_t e, const char* where);   // records text, retur
         if (e__ != cudaSuccess) return ::hts::cuda_fail(e__, name);           \
     } while (0)
 
+// Programmatic dependent launch: the kernel may begin (prologue, weight loads) while its
+// predecessor on the stream drains; it must execute pdl_wait() before touching anything the
+// predecessor wrote or still reads, and calls pdl_trigger() only after that wait, so that "my
+// wait has passed" implies "everything two kernels back is complete" along the whole chain.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 inline int conv_out(int extent, int k, int s) { return (extent - k) / s + 1; }
 
 // Geometry of the fixed four-layer network for one observation shape.

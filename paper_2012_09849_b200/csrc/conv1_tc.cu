@@ -88,6 +88,8 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = tmem_slot;
+    pdl_wait();                                          // frames and the output buffer belong to earlier kernels until here
+    pdl_trigger();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -275,8 +277,8 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
     int grid = sm_count * (per_sm < 1 ? 1 : per_sm);
     if (grid > units) grid = units;
     Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
-    conv1_tc_kernel<<<grid, kThreads, pl.smem_bytes, s>>>(weight_map, p);
-    HTS_LAUNCH_CHECK("conv1_tc_kernel");
+    HTS_CUDA(launch_pdl(conv1_tc_kernel, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
+    note_launch();
     return HTS_OK;
 }
 

@@ -63,10 +63,15 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_d = tmem_slot;
 
+    if (warp == 0 && lane == 0) {                        // the filter does not depend on the previous kernel
+        mbar_arrive_expect_tx(&w_bar, w_bytes);
+        for (int g = 0; g < TAPS * CPT; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+    }
+    pdl_wait();
+    pdl_trigger();
+
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(&w_bar, w_bytes);
-            for (int g = 0; g < TAPS * CPT; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
             int it = 0;
             for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it) {
                 const int b = it % NST;
@@ -179,8 +184,8 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
     }
     const int tiles = (p.total_rows + 127) / 128;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    conv_res_kernel<TAPS, CPT, NST><<<grid, kThreads, smem, s>>>(act_map, weight_map, p);
-    HTS_LAUNCH_CHECK("conv_res_kernel");
+    HTS_CUDA(launch_pdl(conv_res_kernel<TAPS, CPT, NST>, dim3(grid), dim3(kThreads), (size_t)smem, s, act_map, weight_map, p));
+    note_launch();
     return HTS_OK;
 }
 

@@ -75,6 +75,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
         const int total4 = (A + 1) * (kHidden / 4);
         for (int i = threadIdx.x; i < total4; i += 256) s_w4[i] = src[i];
     }
+    pdl_wait();                                        // the head weights above are older than the previous kernel
+    pdl_trigger();
     __syncthreads();
     const float* sw = reinterpret_cast<const float*>(s_w4);
     for (int e = blockIdx.x * 8 + wib; e < n; e += gridDim.x * 8) {
@@ -191,11 +193,10 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
     }
     int blocks = (n + 7) / 8;
     if (blocks > 2 * sm_count) blocks = 2 * sm_count;
-    heads_kernel<<<blocks, 256, smem, s>>>(h_partials, num_splits, split_stride, fc_bias, whead, bhead, A,
-                                           env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu),
-                                           (uint32_t)(seed >> 32), n, actions, logp, values, entropy,
-                                           logits, h_out);
-    HTS_LAUNCH_CHECK("heads_kernel");
+    HTS_CUDA(launch_pdl(heads_kernel, dim3(blocks), dim3(256), smem, s, h_partials, num_splits, split_stride, fc_bias, whead,
+                        bhead, A, env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), n, actions,
+                        logp, values, entropy, logits, h_out));
+    note_launch();
     return HTS_OK;
 }
 

@@ -92,6 +92,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_slot;
+    pdl_wait();
+    pdl_trigger();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -273,8 +275,8 @@ hts_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPar
         HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         attr_set = true;
     }
-    gemm_tc_kernel<BN, EPI><<<grid, 192, smem, s>>>(a, b, p);
-    HTS_LAUNCH_CHECK("gemm_tc_kernel");
+    HTS_CUDA(launch_pdl(gemm_tc_kernel<BN, EPI>, grid, dim3(192), (size_t)smem, s, a, b, p));
+    note_launch();
     return HTS_OK;
 }
 
