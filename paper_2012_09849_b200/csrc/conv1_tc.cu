@@ -8,11 +8,13 @@
 // m = y*Ws + x of the 128-row MMA tile is pixel (y, x) of the band; x = Ws-1 and rows past the
 // band are computed and thrown away.
 //
-// Stages per unit: bulk copies (cp.async.bulk, one per channel) bring the band's uint8 rows
-// into a two-deep ring; four warps convert them to fp16 (bytes 0..255 are exact in fp16; the
-// 1/255 is folded into the accumulator scale) and write the tile; one thread issues
-// 16 * planes tcgen05.mma (128 x 32 x 16) into tensor memory; the same four warps read the
-// accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
+// A CTA is a pipeline of four roles over its units: one thread issues bulk copies
+// (cp.async.bulk, one per channel) of the band's uint8 rows into a ring of staged bands; eight
+// warps turn a staged band into fp16 (a zero-extended byte is the fp16 subnormal b * 2^-24, exact;
+// 2^24 / 255 is folded into the accumulator scale) and write one of two tile buffers; one thread issues 16 * planes
+// tcgen05.mma (128 x 32 x 16) into one of two accumulators in tensor memory; four more warps read
+// an accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
+// Wide inputs (many planes) fall back to one tile buffer and two staged bands to fit.
 #include "conv1_tc.cuh"
 #include "tc_ptx.cuh"
 
@@ -21,7 +23,9 @@ using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 160;                   // warp 0: copies + MMA issue, warps 1..4: convert + epilogue
+constexpr int kThreads = 448;                   // warp 0 copies, warp 1 MMA issue, warps 2..9 convert, warps 10..13 epilogue
+constexpr int kConverters = 256;
+constexpr int kMaxU8 = 3;
 constexpr int kWorkers = 128;
 constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x 128 bytes
 
@@ -35,25 +39,22 @@ struct Conv1Params {
     int* status;
 };
 
-// four bytes -> four fp16 values (b0,b1 | b2,b3), exact: 0x64xx is 1024 + xx
+// Four bytes -> four fp16 values without arithmetic: a byte b zero-extended to 16 bits is the fp16
+// subnormal b * 2^-24, which the tensor core multiplies exactly; the 2^24 goes into the accumulator scale.
 __device__ __forceinline__ void u8x4_to_h4(uint32_t w, uint32_t& lo, uint32_t& hi)
 {
-    const uint32_t magic = 0x64646464u;
-    uint32_t a = __byte_perm(w, magic, 0x4140);         // {b0, 0x64, b1, 0x64} as two halves 0x64b0, 0x64b1
-    uint32_t b = __byte_perm(w, magic, 0x4342);
-    const __half2 k = __half2half2(__ushort_as_half((unsigned short)0x6400));
-    __half2 ha = __hsub2(*reinterpret_cast<__half2*>(&a), k);
-    __half2 hb = __hsub2(*reinterpret_cast<__half2*>(&b), k);
-    lo = *reinterpret_cast<uint32_t*>(&ha);
-    hi = *reinterpret_cast<uint32_t*>(&hb);
+    lo = __byte_perm(w, 0u, 0x4140);                    // {b0, 0, b1, 0}
+    hi = __byte_perm(w, 0u, 0x4342);                    // {b2, 0, b3, 0}
 }
 
+template <int CPT>
 __global__ void __launch_bounds__(kThreads)
 conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
 {
     const Conv1Plan& pl = p.pl;
+    static_assert(CPT == 1 || CPT == 2 || CPT == 4, "planes per tap");
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, u8_full[2], u8_empty[2], a_ready, d_full;
+    __shared__ uint64_t w_bar, u8_full[kMaxU8], u8_empty[kMaxU8], tile_full[2], tile_empty[2], d_full[2], d_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float s_bias[32];
@@ -62,11 +63,13 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     const int plane_bytes = pl.tile_rows * 128;
-    const int w_bytes = 4 * pl.cpt * kChunkBytes;
-    // layout: [weights][fp16 tile: cpt planes][u8 stage 0][u8 stage 1]
+    const int tile_bytes = CPT * plane_bytes;
+    const int w_bytes = 4 * CPT * kChunkBytes;
+    const int NT = pl.tile_bufs, NU = pl.u8_stages;
+    // layout: [weights][fp16 tiles: NT x cpt planes][u8 stages: NU]
     uint8_t* s_w = sm;
     uint8_t* s_tile = sm + w_bytes;
-    uint8_t* s_u8 = s_tile + pl.cpt * plane_bytes;
+    uint8_t* s_u8 = s_tile + NT * tile_bytes;
     const uint32_t a_w = base, a_tile = base + w_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -75,15 +78,17 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
 
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kWorkers); }
-        mbar_init(&a_ready, kWorkers);
-        mbar_init(&d_full, 1);
+        for (int s = 0; s < kMaxU8; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kConverters); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&tile_full[s], kConverters); mbar_init(&tile_empty[s], 1);
+            mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], kWorkers);
+        }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmW);
     }
-    if (threadIdx.x >= 32 && threadIdx.x < 64) s_bias[threadIdx.x - 32] = p.bias[threadIdx.x - 32];
-    if (warp == 0) tmem_alloc(&tmem_slot, 32);
+    if (threadIdx.x >= 64 && threadIdx.x < 96) s_bias[threadIdx.x - 64] = p.bias[threadIdx.x - 64];
+    if (warp == 1) tmem_alloc(&tmem_slot, 64);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -92,16 +97,14 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     pdl_trigger();
 
     if (warp == 0) {
+        // ---- copies: weights once, then each unit's uint8 rows, NU units ahead
         if (lane == 0) {
-            // weights once
             mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
-            for (int g = 0; g < 4 * pl.cpt; ++g) tma_load_2d(s_w + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
-            constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
-            bool alive = true;
-            // software pipeline: the copy of unit i+1 is issued before the MMAs of unit i
-            auto issue_copy = [&](int it, int u) -> bool {
-                const int s = it & 1;
-                if (!mbar_wait(&u8_empty[s], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 11)) return false;
+            for (int g = 0; g < 4 * CPT; ++g) tma_load_2d(s_w + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+            int it = 0;
+            for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
+                const int s = it % NU;
+                if (!mbar_wait(&u8_empty[s], (((uint32_t)(it / NU)) & 1u) ^ 1u, abortp, p.status, 11)) break;
                 const int env = u / pl.bands, band = u - env * pl.bands;
                 const int r0 = 4 * band * pl.R;
                 int rows = pl.H - r0; rows = rows > band_in_rows ? band_in_rows : rows;
@@ -111,79 +114,95 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 uint8_t* dst = s_u8 + s * pl.u8_stage_bytes;
                 for (int c = 0; c < pl.C; ++c)
                     bulk_load(dst + c * band_in_rows * pl.W, src + (size_t)c * pl.H * pl.W, bytes, &u8_full[s]);
-                return true;
-            };
-            int it = 0;
-            int u = blockIdx.x;
-            if (u < units) alive = issue_copy(0, u);
-            if (alive) alive = mbar_wait(&w_bar, 0, abortp, p.status, 12);
-            for (; alive && u < units; u += gridDim.x, ++it) {
-                const int un = u + gridDim.x;
-                if (un < units) { if (!issue_copy(it + 1, un)) break; }
-                if (!mbar_wait(&a_ready, (uint32_t)it & 1u, abortp, p.status, 13)) break;
-                tc_fence_after();
-                uint32_t first = 1;
-                for (int tap = 0; tap < 4; ++tap) {
-                    const int shift = (tap >> 1) * pl.Ws + (tap & 1);
-                    for (int pln = 0; pln < pl.cpt; ++pln) {
-                        const uint64_t adesc = smem_desc_sw128(a_tile + pln * plane_bytes + shift * 128);
-                        const uint64_t bdesc = smem_desc_sw128(a_w + (tap * pl.cpt + pln) * kChunkBytes);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            mma_f16_ss(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, first ? 0u : 1u);
-                            first = 0;
-                        }
-                    }
-                }
-                mma_commit(&d_full);
             }
         }
-    } else {
-        const int tid = threadIdx.x - 32;                // 0..127
-        const int q = warp & 3;                          // TMEM lane quarter this warp may read
-        const int row = q * 32 + lane;                   // tile row handled in the epilogue
-        const float inv = *p.inv_scale;
-        // convert: thread owns one 16-byte chunk position qq of every 16th pixel
-        const int qq = tid & 7, slot = tid >> 3;
+    } else if (warp == 1) {
+        // ---- MMA issue
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
+            bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 12);
+            int it = 0;
+            for (int u = blockIdx.x; alive && u < units; u += gridDim.x, ++it) {
+                const int tb = it % NT, db = it & 1;
+                if (!mbar_wait(&tile_full[tb], ((uint32_t)(it / NT)) & 1u, abortp, p.status, 13)) break;
+                if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 16)) break;
+                tc_fence_after();
+                const uint32_t t_addr = a_tile + tb * tile_bytes;
+                uint32_t acc = 0;
+#pragma unroll
+                for (int tap = 0; tap < 4; ++tap) {
+                    const int shift = (tap >> 1) * pl.Ws + (tap & 1);
+#pragma unroll
+                    for (int pln = 0; pln < CPT; ++pln) {
+                        const uint64_t adesc = smem_desc_sw128(t_addr + pln * plane_bytes + shift * 128);
+                        const uint64_t bdesc = smem_desc_sw128(a_w + (tap * CPT + pln) * kChunkBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) { mma_f16_ss(tmem_d + db * 32, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
+                    }
+                }
+                mma_commit(&tile_empty[tb]);
+                mma_commit(&d_full[db]);
+            }
+        }
+    } else if (warp < 10) {
+        // ---- convert: thread owns 16-byte chunk position qq of every 32nd pixel of a plane
+        const int tid = threadIdx.x - 64;                // 0..255
+        const int qq = tid & 7, slot = tid >> 3;         // slot 0..31
         const int src_q = ((qq >> 1) * band_in_rows + 2 * (qq & 1)) * pl.W;     // channel (qq>>1) of a plane, row pair (qq&1)
         const int plane_src = 4 * band_in_rows * pl.W;                          // four channels per plane
-        const int ey = row / pl.Ws, ex = row - ey * pl.Ws;                       // epilogue pixel of this thread
+        const int ys0 = slot / pl.Ws, xs0 = slot - ys0 * pl.Ws;                  // first pixel of this thread
+        const int dys = 32 / pl.Ws, dxs = 32 - dys * pl.Ws;                      // step of 32 pixels on the grid
         int it = 0;
         for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
-            const int s = it & 1;
-            const int env = u / pl.bands, band = u - env * pl.bands;
-            const int y0 = band * pl.R;
-            int in_rows = pl.H - 4 * y0; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
+            const int s = it % NU, tb = it % NT;
+            const int band = u % pl.bands;
+            int in_rows = pl.H - 4 * band * pl.R; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
             const int pixels = (in_rows >> 2) * pl.Ws;   // space-to-depth pixels present in this band
-            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)it >> 1) & 1u, abortp, p.status, 14)) break;
+            if (!mbar_wait_warp(&tile_empty[tb], (((uint32_t)(it / NT)) & 1u) ^ 1u, abortp, p.status, 17)) break;
+            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 14)) break;
             const uint8_t* src = s_u8 + s * pl.u8_stage_bytes + src_q;
-            for (int pln = 0; pln < pl.cpt; ++pln) {
-                uint8_t* dplane = s_tile + pln * plane_bytes;
+            uint8_t* tile = s_tile + tb * tile_bytes;
+#pragma unroll
+            for (int pln = 0; pln < CPT; ++pln) {
+                uint8_t* dplane = tile + pln * plane_bytes;
                 const uint8_t* splane = src + pln * plane_src;
-                int ys = 0, xs = slot;
-                while (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
-                for (int ps = slot; ps < pixels; ps += 16) {
+                int ys = ys0, xs = xs0;
+#pragma unroll 5
+                for (int ps = slot; ps < pixels; ps += 32) {
                     const uint8_t* s0 = splane + (4 * ys) * pl.W + 4 * xs;
                     const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
                     const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
                     uint4 o;
                     u8x4_to_h4(w0, o.x, o.y);
                     u8x4_to_h4(w1, o.z, o.w);
+                    // chunk qq of row ps, 128-byte swizzle: qq ^ (ps % 8)
                     *reinterpret_cast<uint4*>(dplane + ps * 128 + ((qq ^ (ps & 7)) << 4)) = o;
-                    xs += 16;
-                    while (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
+                    xs += dxs; ys += dys;
+                    if (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
                 }
             }
             fence_async_proxy();                         // tile stores -> visible to the tensor core's reads
             mbar_arrive(&u8_empty[s]);
-            mbar_arrive(&a_ready);
-            // ---- epilogue
-            if (!mbar_wait_warp(&d_full, (uint32_t)it & 1u, abortp, p.status, 15)) break;
+            mbar_arrive(&tile_full[tb]);
+        }
+    } else {
+        // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const float inv = *p.inv_scale;
+        const int ey = row / pl.Ws, ex = row - ey * pl.Ws;
+        int it = 0;
+        for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
+            const int db = it & 1;
+            const int env = u / pl.bands, band = u - env * pl.bands;
+            const int y0 = band * pl.R;
+            if (!mbar_wait_warp(&d_full[db], ((uint32_t)it >> 1) & 1u, abortp, p.status, 15)) break;
             tc_fence_after();
             uint32_t v[32];
-            tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16), v);
+            tmem_ld_32x32(tmem_d + db * 32 + ((uint32_t)(q * 32) << 16), v);
             tmem_ld_wait();
             tc_fence_before();
+            mbar_arrive(&d_empty[db]);
             const int yy = y0 + ey;
             if (ey < pl.R && yy < pl.H1 && ex < pl.W1) {
                 __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (ex >> 1)) * 128 +
@@ -212,7 +231,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_d, 32);
+    if (warp == 1) tmem_dealloc(tmem_d, 64);
 }
 
 __global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int C,
@@ -231,18 +250,23 @@ __global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* _
 
 bool conv1_plan(const Geometry& g, Conv1Plan* pl)
 {
-    if (g.C % 4 || g.H % 4 || g.W % 4) return false;    // bulk copies then start and end on 16-byte boundaries
+    if (g.C % 4 || g.H % 4 || g.W % 4 || (g.C != 4 && g.C != 8 && g.C != 16)) return false;    // bulk copies then start and end on 16-byte boundaries
     pl->C = g.C; pl->H = g.H; pl->W = g.W;
     pl->Hs = g.H / 4; pl->Ws = g.W / 4; pl->Cs = 16 * g.C;
     pl->H1 = pl->Hs - 1; pl->W1 = pl->Ws - 1;
-    if (pl->H1 != g.H1 || pl->W1 != g.W1 || pl->Ws > 64 || pl->H1 < 1) return false;
+    if (pl->H1 != g.H1 || pl->W1 != g.W1 || pl->Ws > 64 || pl->Ws < 3 || pl->H1 < 1) return false;
     pl->cpt = pl->Cs / 64;
     const int rmax = 128 / pl->Ws;
     pl->bands = (pl->H1 + rmax - 1) / rmax;
     pl->R = (pl->H1 + pl->bands - 1) / pl->bands;
     pl->tile_rows = (128 + pl->Ws + 1 + 7) / 8 * 8;
     pl->u8_stage_bytes = (g.C * 4 * (pl->R + 1) * g.W + 127) / 128 * 128;
-    pl->smem_bytes = 1024 + 4 * pl->cpt * kChunkBytes + pl->cpt * pl->tile_rows * 128 + 2 * pl->u8_stage_bytes;
+    const int fixed = 1024 + 4 * pl->cpt * kChunkBytes;
+    const int tile = pl->cpt * pl->tile_rows * 128;
+    // two tile buffers and three staged bands when two CTAs still fit an SM, else the smallest pipeline
+    pl->tile_bufs = 2; pl->u8_stages = 3;
+    if (fixed + 2 * tile + 3 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
+    pl->smem_bytes = fixed + pl->tile_bufs * tile + pl->u8_stages * pl->u8_stage_bytes;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
     return pl->smem_bytes <= 227 * 1024;
 }
@@ -266,18 +290,24 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
         HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
     if (max_smem_set < pl.smem_bytes) {
-        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
         // every kernel of the step asks for the largest shared-memory carve-out, so that the SMs are not
         // re-partitioned between consecutive kernels
-        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<1>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<4>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         max_smem_set = pl.smem_bytes;
     }
-    const int per_sm = (227 * 1024) / (pl.smem_bytes + 1024) > 4 ? 4 : (227 * 1024) / (pl.smem_bytes + 1024);
+    const int per_sm = (227 * 1024) / (pl.smem_bytes + 1024) > 2 ? 2 : (227 * 1024) / (pl.smem_bytes + 1024);
     const int units = n * pl.bands;
     int grid = sm_count * (per_sm < 1 ? 1 : per_sm);
     if (grid > units) grid = units;
     Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
-    HTS_CUDA(launch_pdl(conv1_tc_kernel, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
+    if (pl.cpt == 1) HTS_CUDA(launch_pdl(conv1_tc_kernel<1>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
+    else if (pl.cpt == 2) HTS_CUDA(launch_pdl(conv1_tc_kernel<2>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
+    else HTS_CUDA(launch_pdl(conv1_tc_kernel<4>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
     note_launch();
     return HTS_OK;
 }

@@ -352,7 +352,8 @@ hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s)
         absmax_kernel<<<64, 256, 0, s>>>(bf(m.p), m.n, t->absmax + m.l);
         HTS_LAUNCH_CHECK("absmax");
     }
-    scales_kernel<<<1, 32, 0, s>>>(t->absmax, t->scale, t->inv_scale, 1.0f / 255.0f);
+    // conv1 feeds raw bytes as fp16 subnormals (b * 2^-24): its accumulator scale undoes that and the /255
+    scales_kernel<<<1, 32, 0, s>>>(t->absmax, t->scale, t->inv_scale, 16777216.0f / 255.0f);
     HTS_LAUNCH_CHECK("scales");
     hts_status st1 = conv1_pack_weights(t->pl1, bf(w.conv1_w), t->w1p, t->scale + L_CONV1, s);
     if (st1 != HTS_OK) return st1;
