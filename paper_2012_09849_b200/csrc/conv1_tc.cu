@@ -11,7 +11,7 @@
 // A CTA is a pipeline of four roles over its units: one thread issues bulk copies
 // (cp.async.bulk, one per channel) of the band's uint8 rows into a ring of staged bands; eight
 // warps turn a staged band into fp16 (a zero-extended byte is the fp16 subnormal b * 2^-24, exact;
-// 2^24 / 255 is folded into the accumulator scale) and write one of two tile buffers; one thread issues 16 * planes
+// 2^24 / 255 is folded into the accumulator scale) and write one of three tile buffers; one thread issues 16 * planes
 // tcgen05.mma (128 x 32 x 16) into one of two accumulators in tensor memory; four more warps read
 // an accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
 // Wide inputs (many planes) fall back to one tile buffer and two staged bands to fit.
@@ -25,6 +25,7 @@ namespace {
 
 constexpr int kThreads = 448;                   // warp 0 copies, warp 1 MMA issue, warps 2..9 convert, warps 10..13 epilogue
 constexpr int kConverters = 256;
+constexpr int kMaxTiles = 3;
 constexpr int kMaxU8 = 3;
 constexpr int kWorkers = 128;
 constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x 128 bytes
@@ -54,7 +55,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     const Conv1Plan& pl = p.pl;
     static_assert(CPT == 1 || CPT == 2 || CPT == 4, "planes per tap");
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, u8_full[kMaxU8], u8_empty[kMaxU8], tile_full[2], tile_empty[2], d_full[2], d_empty[2];
+    __shared__ uint64_t w_bar, u8_full[kMaxU8], u8_empty[kMaxU8], tile_full[kMaxTiles], tile_empty[kMaxTiles], d_full[2], d_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float s_bias[32];
@@ -79,10 +80,8 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
         for (int s = 0; s < kMaxU8; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kConverters); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&tile_full[s], kConverters); mbar_init(&tile_empty[s], 1);
-            mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], kWorkers);
-        }
+        for (int s = 0; s < kMaxTiles; ++s) { mbar_init(&tile_full[s], kConverters); mbar_init(&tile_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], kWorkers); }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmW);
@@ -263,9 +262,9 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     pl->u8_stage_bytes = (g.C * 4 * (pl->R + 1) * g.W + 127) / 128 * 128;
     const int fixed = 1024 + 4 * pl->cpt * kChunkBytes;
     const int tile = pl->cpt * pl->tile_rows * 128;
-    // two tile buffers and three staged bands when two CTAs still fit an SM, else the smallest pipeline
-    pl->tile_bufs = 2; pl->u8_stages = 3;
-    if (fixed + 2 * tile + 3 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
+    // three tile buffers and three staged bands when two CTAs still fit an SM, else the smallest pipeline
+    pl->tile_bufs = 3; pl->u8_stages = 3;
+    if (fixed + 3 * tile + 3 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
     pl->smem_bytes = fixed + pl->tile_bufs * tile + pl->u8_stages * pl->u8_stage_bytes;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
     return pl->smem_bytes <= 227 * 1024;
