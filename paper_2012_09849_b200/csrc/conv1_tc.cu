@@ -26,7 +26,7 @@ namespace {
 constexpr int kThreads = 448;                   // warp 0 copies, warp 1 MMA issue, warps 2..9 convert, warps 10..13 epilogue
 constexpr int kConverters = 256;
 constexpr int kMaxTiles = 3;
-constexpr int kMaxU8 = 3;
+constexpr int kMaxU8 = 6;
 constexpr int kWorkers = 128;
 constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x 128 bytes
 
@@ -262,9 +262,9 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     pl->u8_stage_bytes = (g.C * 4 * (pl->R + 1) * g.W + 127) / 128 * 128;
     const int fixed = 1024 + 4 * pl->cpt * kChunkBytes;
     const int tile = pl->cpt * pl->tile_rows * 128;
-    // three tile buffers and three staged bands when two CTAs still fit an SM, else the smallest pipeline
-    pl->tile_bufs = 3; pl->u8_stages = 3;
-    if (fixed + 3 * tile + 3 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
+    // three tile buffers and four staged bands when two CTAs still fit an SM, else the smallest pipeline
+    pl->tile_bufs = 3; pl->u8_stages = 4;
+    if (fixed + 3 * tile + 4 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
     pl->smem_bytes = fixed + pl->tile_bufs * tile + pl->u8_stages * pl->u8_stage_bytes;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
     return pl->smem_bytes <= 227 * 1024;
