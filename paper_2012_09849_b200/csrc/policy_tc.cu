@@ -33,7 +33,7 @@ namespace {
 
 constexpr int BM = 128;                 // rows per tile = TMEM lanes
 constexpr int BK = 64;                  // 16-bit elements per K chunk = one 128-byte swizzle row
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;                 // 3 x 32 KiB: two CTAs per SM, so the 224 FC tiles run in one wave
 constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
 enum { EPI_CONV = 0, EPI_SPLITK = 1 };
 enum { L_CONV1 = 0, L_CONV2, L_CONV3, L_FC, L_COUNT };
