@@ -137,19 +137,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const long m = (long)m0 + r;
             const float inv = *p.inv_scale;
             if (EPI == EPI_SPLITK) {
-                float* dst = p.out_f32 + blockIdx.z * p.split_stride + (size_t)m * p.ldo + n0;
+                // The accumulator arrives one row per thread; a row-per-thread store would touch 32
+                // lines per instruction.  Each warp turns its 32x32 block through shared memory (the
+                // pipeline stages are free by now) so that eight lanes write one full 128-byte line.
+                float* stage = reinterpret_cast<float*>(tiles) + (warp - 2) * (32 * 36);
+                float* dst = p.out_f32 + blockIdx.z * p.split_stride + (size_t)(m0 + q * 32) * p.ldo + n0;
+                const int rl = lane >> 3, c4 = (lane & 7) * 4;
 #pragma unroll
                 for (int c = 0; c < BN; c += 32) {
                     uint32_t v[32];
                     tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
                     tmem_ld_wait();
-                    if (m < p.n_env) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4*>(dst + c + j) =
-                                make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
-                                            __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(stage + lane * 36 + j) =
+                            make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
+                                        __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = 4 * i + rl;
+                        const float4 val = *reinterpret_cast<const float4*>(stage + rr * 36 + c4);
+                        if (m0 + q * 32 + rr < p.n_env) *reinterpret_cast<float4*>(dst + (size_t)rr * p.ldo + c + c4) = val;
                     }
+                    __syncwarp();
                 }
             } else {
                 const int env = (int)(m / p.P_in);
