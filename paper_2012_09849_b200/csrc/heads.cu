@@ -69,44 +69,49 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
 {
     extern __shared__ float4 s_w4[];                   // [(A+1)*512] head weights, staged once per block
     __shared__ float s_out[8][kMaxActions + 1];
+    __shared__ float s_bhead[kMaxActions + 1];
+    __shared__ float4 s_fcb[kHidden / 4];
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
     {
         const float4* src = reinterpret_cast<const float4*>(whead);
         const int total4 = (A + 1) * (kHidden / 4);
         for (int i = threadIdx.x; i < total4; i += 256) s_w4[i] = src[i];
+        // biases too: a global load inside the per-output loop would stall the warp once per iteration
+        if (threadIdx.x <= A) s_bhead[threadIdx.x] = bhead[threadIdx.x];
+        if (fc_bias && threadIdx.x < kHidden / 4) s_fcb[threadIdx.x] = reinterpret_cast<const float4*>(fc_bias)[threadIdx.x];
     }
     pdl_wait();                                        // the head weights above are older than the previous kernel
     pdl_trigger();
     __syncthreads();
-    const float* sw = reinterpret_cast<const float*>(s_w4);
+    const float4* sw4 = s_w4;
     for (int e = blockIdx.x * 8 + wib; e < n; e += gridDim.x * 8) {
-    // hidden vector: split partials summed in index order (four splits' loads in flight at a time)
-    float h[kHidden / 32];
+    const uint32_t env = (uint32_t)env_ids[e];                         // issued early: needed only by the sampler
+    const uint32_t tt = (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
+    // hidden vector: lane l owns units 128*i + 4*l + {0..3}, i = 0..3 (float4 everywhere); split
+    // partials are summed in index order
+    float4 h[4];
+    {
+        const float4* hp = reinterpret_cast<const float4*>(h_partials + (size_t)e * kHidden) + lane;
+        const size_t stride4 = split_stride / 4;
+        float4 part[kMaxSplits][4];
 #pragma unroll
-    for (int i = 0; i < kHidden / 32; ++i) h[i] = 0.f;
+        for (int sp = 0; sp < kMaxSplits; ++sp)
 #pragma unroll
-    for (int sp0 = 0; sp0 < kMaxSplits; sp0 += 4) {
-        if (sp0 < num_splits) {
-            float part[4][kHidden / 32];
+            for (int i = 0; i < 4; ++i)
+                part[sp][i] = (sp < num_splits) ? hp[sp * stride4 + 32 * i] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+        for (int i = 0; i < 4; ++i) {
+            float4 v = part[0][i];
 #pragma unroll
-                for (int i = 0; i < kHidden / 32; ++i)
-                    part[j][i] = (sp0 + j < num_splits)
-                                     ? h_partials[(sp0 + j) * split_stride + (size_t)e * kHidden + lane + 32 * i] : 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int i = 0; i < kHidden / 32; ++i)
-                    if (sp0 + j < num_splits) h[i] = (sp0 + j == 0) ? part[j][i] : h[i] + part[j][i];
+            for (int sp = 1; sp < kMaxSplits; ++sp)
+                if (sp < num_splits) { v.x += part[sp][i].x; v.y += part[sp][i].y; v.z += part[sp][i].z; v.w += part[sp][i].w; }
+            if (fc_bias) {
+                const float4 bb = s_fcb[32 * i + lane];
+                v.x = fmaxf(v.x + bb.x, 0.f); v.y = fmaxf(v.y + bb.y, 0.f); v.z = fmaxf(v.z + bb.z, 0.f); v.w = fmaxf(v.w + bb.w, 0.f);
+            }
+            h[i] = v;
+            if (h_out) reinterpret_cast<float4*>(h_out + (size_t)e * kHidden)[32 * i + lane] = v;
         }
-    }
-#pragma unroll
-    for (int i = 0; i < kHidden / 32; ++i) {
-        float v = h[i];
-        if (fc_bias) { v += fc_bias[lane + 32 * i]; v = v > 0.f ? v : 0.f; }
-        h[i] = v;
-        if (h_out) h_out[(size_t)e * kHidden + lane + 32 * i] = v;
     }
     for (int o0 = 0; o0 <= A; o0 += 4) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -114,7 +119,11 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
         for (int j = 0; j < 4; ++j) {
             const int o = (o0 + j <= A) ? o0 + j : A;
 #pragma unroll
-            for (int i = 0; i < kHidden / 32; ++i) acc[j] = fmaf(sw[o * kHidden + lane + 32 * i], h[i], acc[j]);
+            for (int i = 0; i < 4; ++i) {
+                const float4 w = sw4[o * (kHidden / 4) + 32 * i + lane];
+                acc[j] = fmaf(w.x, h[i].x, acc[j]); acc[j] = fmaf(w.y, h[i].y, acc[j]);
+                acc[j] = fmaf(w.z, h[i].z, acc[j]); acc[j] = fmaf(w.w, h[i].w, acc[j]);
+            }
         }
 #pragma unroll
         for (int m = 16; m > 0; m >>= 1)
@@ -122,7 +131,7 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
             for (int j = 0; j < 4; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], m);
         if (lane < 4 && o0 + lane <= A) {
             const float mine = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
-            s_out[wib][o0 + lane] = mine + bhead[o0 + lane];
+            s_out[wib][o0 + lane] = mine + s_bhead[o0 + lane];
         }
     }
     __syncwarp();
@@ -140,8 +149,6 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
     for (int a = lane; a < A; a += 32) { const float lp = lg[a] - lse; ent -= expf(lp) * lp; }
     ent = warp_sum(ent);
 
-    const uint32_t env = (uint32_t)env_ids[e];
-    const uint32_t tt = (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
     float best = -INFINITY; int best_a = 0x7fffffff;
     for (int a = lane; a < A; a += 32) {
         const float u = action_uniform(env, tt, a, key0, key1);
