@@ -146,6 +146,30 @@ def run_reference(args) -> None:
 
 
 # ------------------------------------------------------------------------------------------------
+def run_ncu_case(steps: int) -> None:
+    """A few actor steps of the bench workload (n = N rows each) and one GAE over [T, N]: the small case
+    that is captured under ncu.  Device footprint: two observation batches and the context (< 0.2 GB)."""
+    import torch
+    import paper_2012_09849_b200 as hts
+    cfg = wl.CONFIGS[WORKLOAD]
+    T, N = cfg.T, cfg.N
+    ctx = hts.hts_policy_create(cfg.C, cfg.H, cfg.W, cfg.A, hts.HTS_DTYPE_BF16, N)
+    hts.hts_policy_load_weights(ctx, hts.weights_to_device(wl.make_weights(cfg), hts.HTS_DTYPE_BF16))
+    obs = [torch.from_numpy(wl.make_obs(cfg, N, batch_index=i)).cuda() for i in range(2)]
+    ids = torch.arange(N, dtype=torch.int32, device="cuda")
+    act = torch.empty(N, dtype=torch.int32, device="cuda")
+    f = [torch.empty(N, device="cuda") for _ in range(3)]
+    for t in range(steps):
+        hts.hts_policy_step(ctx, obs[t % 2], ids, None, t, SEED, N, act, *f)
+    r, v, d, b = (torch.from_numpy(x).cuda() for x in wl.make_rollout(cfg))
+    adv, ret = torch.empty_like(v), torch.empty_like(v)
+    hts.hts_gae(r, v, d, b, cfg.gamma, cfg.lam, T, N, adv, ret)
+    torch.cuda.synchronize()
+    hts.hts_policy_destroy(ctx)
+    print("ncu case done:", steps, "steps")
+
+
+# ------------------------------------------------------------------------------------------------
 def run_ours(args) -> None:
     import torch
     import paper_2012_09849_b200 as hts
@@ -379,8 +403,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ncu-case", type=int, default=0, metavar="STEPS",
+                    help="profiling driver: run STEPS actor steps of the bench workload plus one GAE and exit "
+                         "(no timing; for use under ncu)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.ncu_case > 0:
+        run_ncu_case(args.ncu_case)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
