@@ -11,7 +11,7 @@
 // A CTA is a pipeline of four roles over its units: one thread issues bulk copies
 // (cp.async.bulk, one per channel) of the band's uint8 rows into a ring of staged bands; eight
 // warps turn a staged band into fp16 (a zero-extended byte is the fp16 subnormal b * 2^-24, exact;
-// 2^24 / 255 is folded into the accumulator scale) and write one of three tile buffers; one thread issues 16 * planes
+// 2^24 / 255 is folded into the accumulator scale) and write a ring of 64-channel planes (three or four); one thread issues 16 * planes
 // tcgen05.mma (128 x 32 x 16) into one of two accumulators in tensor memory; four more warps read
 // an accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
 // Wide inputs (many planes) fall back to one tile buffer and two staged bands to fit.
@@ -25,7 +25,7 @@ namespace {
 
 constexpr int kThreads = 448;                   // warp 0 copies, warp 1 MMA issue, warps 2..9 convert, warps 10..13 epilogue
 constexpr int kConverters = 256;
-constexpr int kMaxTiles = 3;
+constexpr int kMaxPlanes = 4;
 constexpr int kMaxU8 = 6;
 constexpr int kWorkers = 128;
 constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x 128 bytes
@@ -55,7 +55,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     const Conv1Plan& pl = p.pl;
     static_assert(CPT == 1 || CPT == 2 || CPT == 4, "planes per tap");
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, u8_full[kMaxU8], u8_empty[kMaxU8], tile_full[kMaxTiles], tile_empty[kMaxTiles], d_full[2], d_empty[2];
+    __shared__ uint64_t w_bar, u8_full[kMaxU8], u8_empty[kMaxU8], plane_full[kMaxPlanes], plane_empty[kMaxPlanes], d_full[2], d_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float s_bias[32];
@@ -64,13 +64,12 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     const int plane_bytes = pl.tile_rows * 128;
-    const int tile_bytes = CPT * plane_bytes;
     const int w_bytes = 4 * CPT * kChunkBytes;
-    const int NT = pl.tile_bufs, NU = pl.u8_stages;
-    // layout: [weights][fp16 tiles: NT x cpt planes][u8 stages: NU]
+    const int NP = pl.plane_bufs, NU = pl.u8_stages;
+    // layout: [weights][ring of NP fp16 planes (64 channels of a band each)][u8 stages: NU]
     uint8_t* s_w = sm;
     uint8_t* s_tile = sm + w_bytes;
-    uint8_t* s_u8 = s_tile + NT * tile_bytes;
+    uint8_t* s_u8 = s_tile + NP * plane_bytes;
     const uint32_t a_w = base, a_tile = base + w_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -80,7 +79,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
         for (int s = 0; s < kMaxU8; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kConverters); }
-        for (int s = 0; s < kMaxTiles; ++s) { mbar_init(&tile_full[s], kConverters); mbar_init(&tile_empty[s], 1); }
+        for (int s = 0; s < kMaxPlanes; ++s) { mbar_init(&plane_full[s], kConverters); mbar_init(&plane_empty[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], kWorkers); }
         abort_flag = 0;
         fence_barrier_init();
@@ -120,27 +119,29 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
             bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 12);
-            int it = 0;
+            int it = 0, pb = 0;
+            uint32_t pph = 0;
             for (int u = blockIdx.x; alive && u < units; u += gridDim.x, ++it) {
-                const int tb = it % NT, db = it & 1;
-                if (!mbar_wait(&tile_full[tb], ((uint32_t)(it / NT)) & 1u, abortp, p.status, 13)) break;
+                const int db = it & 1;
                 if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 16)) break;
-                tc_fence_after();
-                const uint32_t t_addr = a_tile + tb * tile_bytes;
                 uint32_t acc = 0;
 #pragma unroll
-                for (int tap = 0; tap < 4; ++tap) {
-                    const int shift = (tap >> 1) * pl.Ws + (tap & 1);
+                for (int pln = 0; pln < CPT; ++pln) {     // planes arrive one by one: MMAs of plane k overlap the conversion of k+1
+                    if (!mbar_wait(&plane_full[pb], pph, abortp, p.status, 13)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t p_addr = a_tile + pb * plane_bytes;
 #pragma unroll
-                    for (int pln = 0; pln < CPT; ++pln) {
-                        const uint64_t adesc = smem_desc_sw128(t_addr + pln * plane_bytes + shift * 128);
+                    for (int tap = 0; tap < 4; ++tap) {
+                        const int shift = (tap >> 1) * pl.Ws + (tap & 1);
+                        const uint64_t adesc = smem_desc_sw128(p_addr + shift * 128);
                         const uint64_t bdesc = smem_desc_sw128(a_w + (tap * CPT + pln) * kChunkBytes);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) { mma_f16_ss(tmem_d + db * 32, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
                     }
+                    mma_commit(&plane_empty[pb]);
+                    if (++pb == NP) { pb = 0; pph ^= 1u; }
                 }
-                mma_commit(&tile_empty[tb]);
-                mma_commit(&d_full[db]);
+                if (alive) mma_commit(&d_full[db]);
             }
         }
     } else if (warp < 10) {
@@ -151,19 +152,20 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         const int plane_src = 4 * band_in_rows * pl.W;                          // four channels per plane
         const int ys0 = slot / pl.Ws, xs0 = slot - ys0 * pl.Ws;                  // first pixel of this thread
         const int dys = 32 / pl.Ws, dxs = 32 - dys * pl.Ws;                      // step of 32 pixels on the grid
-        int it = 0;
-        for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
-            const int s = it % NU, tb = it % NT;
+        int it = 0, pb = 0;
+        uint32_t pph = 0;
+        bool alive = true;
+        for (int u = blockIdx.x; alive && u < units; u += gridDim.x, ++it) {
+            const int s = it % NU;
             const int band = u % pl.bands;
             int in_rows = pl.H - 4 * band * pl.R; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
             const int pixels = (in_rows >> 2) * pl.Ws;   // space-to-depth pixels present in this band
-            if (!mbar_wait_warp(&tile_empty[tb], (((uint32_t)(it / NT)) & 1u) ^ 1u, abortp, p.status, 17)) break;
             if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 14)) break;
             const uint8_t* src = s_u8 + s * pl.u8_stage_bytes + src_q;
-            uint8_t* tile = s_tile + tb * tile_bytes;
 #pragma unroll
             for (int pln = 0; pln < CPT; ++pln) {
-                uint8_t* dplane = tile + pln * plane_bytes;
+                if (!mbar_wait_warp(&plane_empty[pb], pph ^ 1u, abortp, p.status, 17)) { alive = false; break; }
+                uint8_t* dplane = s_tile + pb * plane_bytes;
                 const uint8_t* splane = src + pln * plane_src;
                 int ys = ys0, xs = xs0;
 #pragma unroll 5
@@ -179,10 +181,11 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                     xs += dxs; ys += dys;
                     if (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
                 }
+                fence_async_proxy();                     // plane stores -> visible to the tensor core's reads
+                mbar_arrive(&plane_full[pb]);
+                if (++pb == NP) { pb = 0; pph ^= 1u; }
             }
-            fence_async_proxy();                         // tile stores -> visible to the tensor core's reads
-            mbar_arrive(&u8_empty[s]);
-            mbar_arrive(&tile_full[tb]);
+            if (alive) mbar_arrive(&u8_empty[s]);
         }
     } else {
         // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1
@@ -261,13 +264,17 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     pl->tile_rows = (128 + pl->Ws + 1 + 7) / 8 * 8;
     pl->u8_stage_bytes = (g.C * 4 * (pl->R + 1) * g.W + 127) / 128 * 128;
     const int fixed = 1024 + 4 * pl->cpt * kChunkBytes;
-    const int tile = pl->cpt * pl->tile_rows * 128;
-    // three tile buffers and four staged bands when two CTAs still fit an SM, else the smallest pipeline
-    pl->tile_bufs = 3; pl->u8_stages = 4;
-    if (fixed + 3 * tile + 4 * pl->u8_stage_bytes > 110 * 1024) { pl->tile_bufs = 1; pl->u8_stages = 2; }
-    pl->smem_bytes = fixed + pl->tile_bufs * tile + pl->u8_stages * pl->u8_stage_bytes;
+    const int plane = pl->tile_rows * 128;
+    // The fp16 planes (64 channels of a band each) form a ring.  Narrow inputs: 3 planes = 3 units in
+    // flight and 4 staged bands, small enough for two CTAs per SM.  Wide inputs: 4 planes, one CTA per SM.
+    pl->plane_bufs = pl->cpt == 1 ? 3 : 4;
+    const int budget = (pl->cpt == 1 ? 110 : 226) * 1024 - fixed - pl->plane_bufs * plane;
+    pl->u8_stages = budget / pl->u8_stage_bytes;
+    if (pl->u8_stages > 4) pl->u8_stages = 4;
+    if (pl->u8_stages < 2) return false;
+    pl->smem_bytes = fixed + pl->plane_bufs * plane + pl->u8_stages * pl->u8_stage_bytes;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
-    return pl->smem_bytes <= 227 * 1024;
+    return true;
 }
 
 hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __half* packed, const float* scale,

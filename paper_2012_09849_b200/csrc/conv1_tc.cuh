@@ -16,7 +16,7 @@ struct Conv1Plan {
     int R, bands;           // output rows per band, bands per environment
     int tile_rows;          // rows allocated per plane of the fp16 tile
     int u8_stage_bytes;     // one staged band of uint8 input
-    int tile_bufs, u8_stages; // fp16 tile buffers (1 or 2) and staged bands (2 or 3)
+    int plane_bufs, u8_stages; // fp16 planes in the ring (3 or 4) and staged bands (2..4)
     int smem_bytes;         // dynamic shared memory of the kernel
     int H1s, W1s, P1s;      // space-to-depth(2) grid of the output (input layout of conv2)
 };
