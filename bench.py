@@ -350,6 +350,32 @@ def run_ours(args) -> None:
                "d2h_bytes_per_step": T * N * 16 + 8 * T * N, "steps": ksteps}
     hts.hts_policy_destroy(ctx)
 
+    # ---- the same actor step at the largest batch of the configurations (cfg5: the whole 8192-env pool,
+    #      4x84x84 frames, 18 actions): how the kernels behave when launch and pipeline-fill costs amortise
+    big = None
+    if rank == 0:
+        c5 = wl.CONFIGS[5]
+        nb = c5.N
+        ctx5 = hts.hts_policy_create(c5.C, c5.H, c5.W, c5.A, hts.HTS_DTYPE_BF16, nb)
+        hts.hts_policy_load_weights(ctx5, hts.weights_to_device(wl.make_weights(c5), hts.HTS_DTYPE_BF16, dev))
+        obs5 = [torch.from_numpy(wl.make_obs(c5, nb, batch_index=i)).to(dev) for i in range(2)]   # 2 x 231 MB > L2
+        ids5 = torch.arange(nb, dtype=torch.int32, device=dev)
+        o5 = [torch.empty(nb, dtype=torch.int32, device=dev)] + [torch.empty(nb, device=dev) for _ in range(3)]
+        for t in range(5):
+            hts.hts_policy_step(ctx5, obs5[t % 2], ids5, None, t, SEED, nb, *o5, None, h_act_stream)
+        a5, b5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 40
+        a5.record(s_act)
+        for t in range(reps):
+            hts.hts_policy_step(ctx5, obs5[t % 2], ids5, None, t, SEED, nb, *o5, None, h_act_stream)
+        b5.record(s_act); torch.cuda.synchronize()
+        us5 = 1e3 * a5.elapsed_time(b5) / reps
+        tf5 = 2.0 * macs_per_env_step(c5) * nb / (us5 * 1e-6) / 1e12
+        big = {"workload": c5.name, "n": nb, "us_per_step": us5, "env_steps_per_s": nb / (us5 * 1e-6), "tflops": tf5,
+               "frac_of_bf16_sustained": tf5 / peak_tf, "frac_of_bf16_burst": tf5 / peaks["bf16_tflops"]}
+        hts.hts_policy_destroy(ctx5)
+        del obs5
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -389,6 +415,8 @@ def run_ours(args) -> None:
         "gae": {"us_cold": gae_us, "elems_per_s": T * N / (gae_us * 1e-6), "gbs_cold": gae_bytes / (gae_us * 1e-6) / 1e9,
                 "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
                          "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
+        "actor_step_us": 1e3 * ms / (args.steps * T),
+        "large_batch_actor_step": big,
         "cpu_baseline": cpu,
     }
     print(json.dumps(out))
