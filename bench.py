@@ -31,6 +31,9 @@ if ROOT not in sys.path:
 import hts_workloads as wl  # noqa: E402
 
 WORKLOAD = 3                       # hts_workloads.CONFIGS index
+# dram__bytes_read.sum + dram__bytes_write.sum of one conv1_tc_kernel<1> launch at this workload (n = 1024),
+# from the ncu capture summarised in profiles/actor_step_cfg3_n1024.md; reported only for that kernel
+CONV1_DRAM_TRAFFIC_BYTES = 28954880 + 39936
 METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
 UNIT = "env-steps/s"
 SEED = 0x5EED
@@ -318,7 +321,9 @@ def run_ours(args) -> None:
     achieved_tf = 2.0 * macs[top] * N / (top_us * 1e-6) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "kernel": top, "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved_tf / peak_tf, "peak_kind": peak_kind + " sustained", "traffic": None,
+                "frac": achieved_tf / peak_tf, "peak_kind": peak_kind + " sustained",
+                "traffic": CONV1_DRAM_TRAFFIC_BYTES if top == "conv1" else None,
+                "algorithmic_bytes": N * obs_bytes if top == "conv1" else None,
                 "us_per_launch": top_us}
     whole_tf = 2.0 * macs_per_env_step(cfg) * value / world / 1e12
 
