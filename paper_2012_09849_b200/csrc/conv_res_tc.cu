@@ -7,9 +7,14 @@
 // per 64-channel plane, 128-byte swizzle) and every tap reads the same tile through a shared-
 // memory descriptor whose start address is moved by `shift` rows: the swizzle is a function of
 // the address bits, so a start that is a multiple of 128 bytes keeps the pattern intact.
-// Activation tiles sit in a 3- or 4-deep ring and the accumulator is double buffered, each
-// buffer with its own four epilogue warps: copies, MMAs and epilogues of different tiles overlap.  Rows whose pixel lies outside the output extent are
-// computed and dropped by the epilogue.
+// Activation tiles sit in a ring; four accumulators live in tensor memory.  Two warps issue MMAs,
+// warp g for the CTA's tiles g, g+2, ... into accumulators g and g+2 in turn, and each accumulator
+// has its own four epilogue warps, so copies, MMAs and epilogues of different tiles overlap.
+// Measured: a 128x64x16 MMA occupies the tensor core for 48 clocks (128 + 64 operand rows of 32
+// bytes from shared memory at 128 bytes per clock), one thread issues one every 70 to 100 clocks,
+// and one epilogue takes about 2300 clocks per tile; two issuers keep the tensor core busy and
+// four epilogue groups keep the issuers from waiting for an accumulator.  Rows whose pixel lies
+// outside the output extent are computed and dropped by the epilogue.
 #include "conv_res_tc.cuh"
 #include "tc_ptx.cuh"
 
@@ -18,7 +23,8 @@ using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 320;                   // warp 0 copies, warp 1 MMA issue, warps 2..5 and 6..9 epilogue
+constexpr int kAcc = 4;                         // accumulators in tensor memory (64 columns each)
+constexpr int kThreads = 128 + kAcc * 128;      // warp 0 copies, warps 1 and 2 issue MMAs, warp 3 idle, then four epilogue warps per accumulator
 constexpr int kChunkBytes = 64 * 128;           // one filter K chunk: 64 output channels x 128 bytes
 
 // 256-bit store of eight packed half2 (one 32-byte sector)
@@ -33,7 +39,7 @@ __global__ void __launch_bounds__(kThreads)
 conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const ConvResParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, a_full[NST], a_empty[NST], d_full[2], d_empty[2];
+    __shared__ uint64_t w_bar, a_full[NST], a_empty[NST], d_full[kAcc], d_empty[kAcc];
     __shared__ float s_bias[64];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -50,14 +56,14 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
         for (int b = 0; b < NST; ++b) { mbar_init(&a_full[b], 1); mbar_init(&a_empty[b], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 128); }
+        for (int b = 0; b < kAcc; ++b) { mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 128); }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmW);
     }
     if (threadIdx.x >= 64 && threadIdx.x < 128) s_bias[threadIdx.x - 64] = p.bias[threadIdx.x - 64];
-    if (warp == 1) tmem_alloc(&tmem_slot, 128);
+    if (warp == 1) tmem_alloc(&tmem_slot, kAcc * 64);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -81,19 +87,20 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int pl = 0; pl < CPT; ++pl) tma_load_2d(dst + pl * plane_bytes, &tmA, pl * 64, tile * 128, &a_full[b]);
             }
         }
-    } else if (warp == 1) {
+    } else if (warp <= 2) {
         if (lane == 0) {
+            // issuing thread g: tiles g, g+2, ... of this CTA, accumulator it % 4 (g, g+2, g, ...)
+            const int g = warp - 1;
             constexpr uint32_t idesc = instr_desc_f16(0, 128, 64);
             bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 22);
-            int it = 0;
-            for (int tile = blockIdx.x; alive && tile < tiles; tile += gridDim.x, ++it) {
-                const int b = it % NST, db = it & 1;
+            int it = g;
+            for (int tile = blockIdx.x + g * gridDim.x; alive && tile < tiles; tile += 2 * gridDim.x, it += 2) {
+                const int b = it % NST, db = it % kAcc;
                 if (!mbar_wait(&a_full[b], ((uint32_t)(it / NST)) & 1u, abortp, p.status, 23)) break;
-                if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 24)) break;
+                if (!mbar_wait(&d_empty[db], (((uint32_t)(it / kAcc)) & 1u) ^ 1u, abortp, p.status, 24)) break;
                 tc_fence_after();
                 const uint32_t a_addr = base + w_bytes + b * a_bytes;
                 const uint32_t d_addr = tmem_d + db * 64;
-                uint32_t acc = 0;
 #pragma unroll
                 for (int tap = 0; tap < TAPS; ++tap) {
 #pragma unroll
@@ -101,26 +108,26 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         const uint64_t adesc = smem_desc_sw128(a_addr + pl * plane_bytes + p.tap_shift[tap] * 128);
                         const uint64_t bdesc = smem_desc_sw128(base + (tap * CPT + pl) * kChunkBytes);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) { mma_f16_ss(d_addr, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
+                        for (int k = 0; k < 4; ++k) mma_f16_ss(d_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (tap | pl | k) != 0);
                     }
                 }
                 mma_commit(&a_empty[b]);
                 mma_commit(&d_full[db]);
             }
         }
-    } else {
-        // two groups of four warps; group g owns accumulator buffer g, i.e. every other tile
-        const int grp = (warp - 2) >> 2;
+    } else if (warp >= 4) {
+        // four warps per accumulator: group j drains accumulator j, i.e. tiles j, j+4, ... of the CTA
+        const int grp = (warp - 4) >> 2;
         const int q = warp & 3;                         // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;
         const float inv = *p.inv_scale;
         int it = grp;
-        for (int tile = blockIdx.x + grp * gridDim.x; tile < tiles; tile += 2 * gridDim.x, it += 2) {
-            if (!mbar_wait_warp(&d_full[grp], ((uint32_t)it >> 1) & 1u, abortp, p.status, 25)) break;
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < tiles; tile += kAcc * gridDim.x, it += kAcc) {
+            if (!mbar_wait_warp(&d_full[grp], ((uint32_t)(it / kAcc)) & 1u, abortp, p.status, 25)) break;
             tc_fence_after();
-            const long m = (long)tile * 128 + r;
-            const int env = (int)(m / p.P_in);
-            const int pix = (int)(m - (long)env * p.P_in);
+            const uint32_t m = (uint32_t)tile * 128u + (uint32_t)r;       // < total_rows + 128, which fits 32 bits
+            const int env = (int)(m / (uint32_t)p.P_in);
+            const int pix = (int)(m - (uint32_t)env * (uint32_t)p.P_in);
             const int y = pix / p.W_in, x = pix - y * p.W_in;
             const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
             __half* dst = p.out + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * 64;
@@ -159,7 +166,7 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_d, 128);
+    if (warp == 1) tmem_dealloc(tmem_d, kAcc * 64);
 }
 
 }  // namespace
@@ -174,7 +181,7 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
         HTS_CUDA(cudaGetDevice(&dev));
         HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
-    constexpr int NST = CPT == 2 ? 3 : 4;        // activation tiles in flight
+    constexpr int NST = CPT == 2 ? 4 : 6;        // activation tiles in the ring: two being multiplied, the rest in flight
     const int smem = 1024 + TAPS * CPT * kChunkBytes + NST * CPT * p.tile_rows * 128;
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;
     if (smem > smem_set) {
