@@ -236,6 +236,241 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     if (warp == 1) tmem_dealloc(tmem_d, 64);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Four-channel frames (Cs = 64): the A operand goes to tensor memory instead of shared memory.
+//
+// The shared-memory kernel above is bound by shared-memory bandwidth: each 128x32x16 MMA fetches
+// 4 KB of A and 1 KB of B (40 clocks at 128 bytes per clock) and every space-to-depth pixel is
+// fetched once per tap.  With tcgen05.mma taking A from tensor memory only B (1 KB) comes from
+// shared memory, and tensor memory has no shifted views, so the converter writes the im2col row
+// of each output pixel (4 taps x 64 channels = 256 fp16 = 128 columns) straight from registers
+// with tcgen05.st.  Rows of a tile are then free to be ANY 128 output pixels: tile t covers pixels
+// [128 t, 128 t + 128) of the batch in (env, y, x) order, no row of the MMA is wasted.
+//
+// One tile: the copy thread brings the input rows under the tile's output rows (at most two
+// environments) into a staged buffer.  A is one buffer of four quarters, one per filter tap
+// (dy,dx), 32 columns each.  Converter warps 2..5 write the dy = 0 quarters, warps 6..9 the dy = 1
+// quarters, each thread its own row.  Two threads issue MMAs, thread h the four K steps of each
+// dy = h quarter as it arrives, into its own accumulator (one thread issues an MMA every 55 to
+// 110 clocks, and MMAs of two threads into one accumulator would have no defined order); the
+// epilogue adds the two in a fixed order.  A quarter is refilled for the next tile as soon as its
+// MMAs are done.  Two CTAs share an SM.
+constexpr int kTsThreads = 480;      // warp 0 copies, 1 and 14 issue, 2..9 convert, 10..13 epilogue
+constexpr int kTsStagesMax = 6;
+
+// (environment, output row, column) of a pixel that advances by a fixed number of pixels per step
+struct PixelWalk {
+    int e, y, x;
+    int sq, sr, eq, er;              // step = sq rows + sr columns; sq rows = eq environments + er rows
+    __device__ void init(uint32_t px, uint32_t step, int H1, int W1)
+    {
+        const uint32_t g = px / (uint32_t)W1;
+        x = (int)(px - g * (uint32_t)W1);
+        e = (int)(g / (uint32_t)H1);
+        y = (int)(g - (uint32_t)e * (uint32_t)H1);
+        sq = (int)(step / (uint32_t)W1); sr = (int)(step - (uint32_t)sq * (uint32_t)W1);
+        eq = sq / H1; er = sq - eq * H1;
+    }
+    __device__ __forceinline__ void advance(int H1, int W1)
+    {
+        x += sr; y += er; e += eq;
+        if (x >= W1) { x -= W1; ++y; }
+        if (y >= H1) { y -= H1; ++e; }
+    }
+};
+
+// rows of the tile that starts at pixel (e0, y0, x0): nA inside e0, nB inside e0 + 1
+__device__ __forceinline__ void ts_rows(const Conv1Plan& pl, int n, int e0, int y0, int x0, int& nA, int& nB)
+{
+    int rows = (x0 + 127) / pl.W1 + 1;
+    const int left_batch = (n - e0) * pl.H1 - y0;            // output rows from here to the end of the batch
+    if (rows > left_batch) rows = left_batch;
+    const int left = pl.H1 - y0;
+    nA = rows < left ? rows : left;
+    nB = rows - nA;
+}
+
+__global__ void __launch_bounds__(kTsThreads, 2)
+conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
+{
+    const Conv1Plan& pl = p.pl;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t w_bar, u8_full[kTsStagesMax], u8_empty[kTsStagesMax], q_full[4], q_empty[4], d_full[2], d_empty[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ float s_bias[32];
+    volatile int* abortp = &abort_flag;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    constexpr int w_bytes = 4 * kChunkBytes;
+    uint8_t* s_u8 = sm + w_bytes;
+    const int NU = pl.ts_stages;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles = (int)(((long)p.n * pl.H1 * pl.W1 + 127) / 128);       // the host keeps n*H1*W1 below 2^31
+    const uint32_t step = 128u * gridDim.x;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&w_bar, 1);
+        for (int s = 0; s < kTsStagesMax; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kConverters); }
+        for (int s = 0; s < 4; ++s) { mbar_init(&q_full[s], kConverters / 2); mbar_init(&q_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 2); mbar_init(&d_empty[s], kWorkers); }
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmW);
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 96) s_bias[threadIdx.x - 64] = p.bias[threadIdx.x - 64];
+    if (warp == 1) tmem_alloc(&tmem_slot, 256);               // columns 0..127 A; 128 + 64 db + 32 h: accumulator h of buffer db
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_a = tmem_slot, tmem_d = tmem_slot + 128;
+    pdl_wait();
+    pdl_trigger();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
+            for (int g = 0; g < 4; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+            const size_t chan = (size_t)pl.H * pl.W, frame = chan * pl.C;
+            PixelWalk first;
+            first.init(128u * blockIdx.x, step, pl.H1, pl.W1);
+            int it = 0;
+            for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, first.advance(pl.H1, pl.W1)) {
+                const int s = it % NU;
+                if (!mbar_wait(&u8_empty[s], (((uint32_t)(it / NU)) & 1u) ^ 1u, abortp, p.status, 31)) break;
+                int nA, nB;
+                ts_rows(pl, p.n, first.e, first.y, first.x, nA, nB);
+                const uint32_t bytesA = (uint32_t)((4 * nA + 4) * pl.W), bytesB = nB ? (uint32_t)((4 * nB + 4) * pl.W) : 0u;
+                mbar_arrive_expect_tx(&u8_full[s], (bytesA + bytesB) * pl.C);
+                // staged layout: channel c at c * ts_chan_bytes; inside it the rows of e0, then the rows of e0 + 1
+                uint8_t* dst = s_u8 + s * pl.ts_stage_bytes;
+                const uint8_t* srcA = p.obs + (size_t)first.e * frame + (size_t)(4 * first.y) * pl.W;
+                for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * pl.ts_chan_bytes, srcA + c * chan, bytesA, &u8_full[s]);
+                if (nB) {
+                    const uint8_t* srcB = p.obs + (size_t)(first.e + 1) * frame;
+                    for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * pl.ts_chan_bytes + bytesA, srcB + c * chan, bytesB, &u8_full[s]);
+                }
+            }
+        }
+    } else if (warp == 1 || warp == 14) {
+        if (lane == 0) {
+            const int h = warp == 1 ? 0 : 1;
+            constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
+            bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 32);
+            int it = 0;
+            for (int tile = blockIdx.x; alive && tile < tiles; tile += gridDim.x, ++it) {
+                const int db = it & 1;
+                if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 33)) break;
+                const uint32_t d_addr = tmem_d + db * 64 + h * 32;
+#pragma unroll
+                for (int dx = 0; dx < 2; ++dx) {
+                    const int qd = 2 * h + dx;                // quarter = filter tap = weight chunk
+                    if (!mbar_wait(&q_full[qd], (uint32_t)it & 1u, abortp, p.status, 34)) { alive = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t bdesc = smem_desc_sw128(base + qd * kChunkBytes) + 2 * k;
+                        mma_f16_ts(d_addr, tmem_a + 32 * qd + 8 * k, bdesc, idesc, (dx | k) != 0);
+                    }
+                    mma_commit(&q_empty[qd]);
+                }
+                if (alive) mma_commit(&d_full[db]);
+            }
+        }
+    } else if (warp < 10) {
+        // ---- convert: thread = row m of the tile; warps 2..5 the dy = 0 quarters, warps 6..9 dy = 1
+        const int h = (warp - 2) >> 2;
+        const int q = warp & 3, m = q * 32 + lane;
+        const uint32_t st_addr = tmem_a + ((uint32_t)(q * 32) << 16) + 64 * h;
+        PixelWalk first, mine;
+        first.init(128u * blockIdx.x, step, pl.H1, pl.W1);
+        mine.init(128u * blockIdx.x + (uint32_t)m, step, pl.H1, pl.W1);
+        int it = 0;
+        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, first.advance(pl.H1, pl.W1), mine.advance(pl.H1, pl.W1)) {
+            const int s = it % NU;
+            const bool valid = mine.e < p.n;
+            // Staged input row under this pixel's window: four rows per output row since the tile's
+            // first one, plus the four extra rows that close the first environment's part.
+            const int segB = mine.e != first.e;
+            const int row = 4 * ((segB ? pl.H1 : 0) + mine.y - first.y + segB + h);
+            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 35)) break;
+            const uint8_t* src = s_u8 + s * pl.ts_stage_bytes + row * pl.W + 4 * mine.x;
+            bool alive = true;
+#pragma unroll
+            for (int dx = 0; dx < 2; ++dx) {
+                uint32_t r[32];
+                const uint8_t* pc = src + 4 * dx;
+#pragma unroll
+                for (int c = 0; c < 4; ++c, pc += pl.ts_chan_bytes) {
+                    const uint8_t* pr = pc;
+#pragma unroll
+                    for (int uy = 0; uy < 4; ++uy, pr += pl.W) {
+                        const uint32_t w = valid ? *reinterpret_cast<const uint32_t*>(pr) : 0u;
+                        u8x4_to_h4(w, r[c * 8 + uy * 2], r[c * 8 + uy * 2 + 1]);
+                    }
+                }
+                if (dx == 1) mbar_arrive(&u8_empty[s]);       // the staged rows are in registers
+                if (!mbar_wait_warp(&q_empty[2 * h + dx], ((uint32_t)it & 1u) ^ 1u, abortp, p.status, 36)) { alive = false; break; }
+                tc_fence_after();
+                tmem_st_32x32(st_addr + 32 * dx, r);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&q_full[2 * h + dx]);
+            }
+            if (!alive) break;
+        }
+    } else if (warp < 14) {
+        // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1
+        const int q = warp & 3, m = q * 32 + lane;
+        const float inv = *p.inv_scale;
+        PixelWalk mine;
+        mine.init(128u * blockIdx.x + (uint32_t)m, step, pl.H1, pl.W1);
+        int it = 0;
+        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, mine.advance(pl.H1, pl.W1)) {
+            const int db = it & 1;
+            if (!mbar_wait_warp(&d_full[db], ((uint32_t)it >> 1) & 1u, abortp, p.status, 37)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_d + db * 64 + ((uint32_t)(q * 32) << 16);
+            __half* dst = p.out + ((size_t)mine.e * pl.P1s + (size_t)(mine.y >> 1) * pl.W1s + (mine.x >> 1)) * 128 +
+                          ((mine.y & 1) * 2 + (mine.x & 1)) * 32;
+#pragma unroll
+            for (int j = 0; j < 32; j += 16) {
+                uint32_t v0[16], v1[16];
+                tmem_ld_32x16(taddr + j, v0);               // dy = 0 taps
+                tmem_ld_32x16(taddr + 32 + j, v1);          // dy = 1 taps
+                tmem_ld_wait();
+                if (j == 16) {
+                    tc_fence_before();
+                    mbar_arrive(&d_empty[db]);
+                }
+                if (mine.e < p.n) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int hh = 0; hh < 8; ++hh) {
+                        const int c = 2 * hh;
+                        const float a0 = __uint_as_float(v0[c]) + __uint_as_float(v1[c]);
+                        const float a1 = __uint_as_float(v0[c + 1]) + __uint_as_float(v1[c + 1]);
+                        __half2 tt = __floats2half2_rn(fmaf(a0, inv, s_bias[j + c]), fmaf(a1, inv, s_bias[j + c + 1]));
+                        tt = __hmin2(__hmax2(tt, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
+                        pk[hh] = *reinterpret_cast<uint32_t*>(&tt);
+                    }
+                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                   "r"(pk[6]), "r"(pk[7]) : "memory");
+                }
+            }
+        }
+    }
+    if (*abortp) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_slot, 256);
+}
+
 __global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int C,
                                   const float* __restrict__ scale)
 {
@@ -274,6 +509,19 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     if (pl->u8_stages < 2) return false;
     pl->smem_bytes = fixed + pl->plane_bufs * plane + pl->u8_stages * pl->u8_stage_bytes;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
+    // tensor-memory variant: four-channel frames whose image has at least one tile of output pixels
+    // (a tile then touches at most two environments)
+    pl->ts = pl->cpt == 1 && pl->H1 * pl->W1 >= 128;
+    if (pl->ts) {
+        const int max_rows = (128 + pl->W1 - 2) / pl->W1 + 1;             // output rows one tile can touch
+        pl->ts_chan_bytes = g.W * (4 * max_rows + 8);                     // one channel of a staged tile (a multiple of 16)
+        pl->ts_stage_bytes = (g.C * pl->ts_chan_bytes + 127) / 128 * 128;
+        int st = (100 * 1024 - 4 * kChunkBytes) / pl->ts_stage_bytes;     // two CTAs per SM
+        if (st > kTsStagesMax) st = kTsStagesMax;
+        if (st < 2) pl->ts = 0;
+        pl->ts_stages = st;
+        pl->ts_smem_bytes = 1024 + 4 * kChunkBytes + st * pl->ts_stage_bytes;
+    }
     return true;
 }
 
@@ -305,6 +553,22 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
         HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<4>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         max_smem_set = pl.smem_bytes;
+    }
+    if (pl.ts && (long)n * pl.H1 * pl.W1 < (1L << 31) - 128 * 2 * sm_count) {
+        static int ts_smem_set = 0;
+        if (ts_smem_set < pl.ts_smem_bytes) {
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.ts_smem_bytes));
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+            ts_smem_set = pl.ts_smem_bytes;
+        }
+        const long total_px = (long)n * pl.H1 * pl.W1;
+        const int tiles = (int)((total_px + 127) / 128);
+        int grid = 2 * sm_count;
+        if (grid > tiles) grid = tiles;
+        Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
+        HTS_CUDA(launch_pdl(conv1_ts_kernel, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
+        note_launch();
+        return HTS_OK;
     }
     const int per_sm = (227 * 1024) / (pl.smem_bytes + 1024) > 2 ? 2 : (227 * 1024) / (pl.smem_bytes + 1024);
     const int units = n * pl.bands;

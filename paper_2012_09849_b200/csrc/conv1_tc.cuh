@@ -19,6 +19,8 @@ struct Conv1Plan {
     int plane_bufs, u8_stages; // fp16 planes in the ring (3 or 4) and staged bands (2..4)
     int smem_bytes;         // dynamic shared memory of the kernel
     int H1s, W1s, P1s;      // space-to-depth(2) grid of the output (input layout of conv2)
+    int ts;                 // 1: the tensor-memory variant applies (four-channel frames)
+    int ts_chan_bytes, ts_stage_bytes, ts_stages, ts_smem_bytes;   // its staged input buffers and shared memory
 };
 
 // false if the geometry does not fit the kernel (C not a multiple of 4, W too wide, ...)
