@@ -257,6 +257,12 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
 // MMAs are done.  Two CTAs share an SM.
 constexpr int kTsThreads = 480;      // warp 0 copies, 1 and 14 issue, 2..9 convert, 10..13 epilogue
 constexpr int kTsStagesMax = 6;
+// bytes of one channel of a staged tile: four input rows per output row a tile can touch, plus the
+// closing rows of two environments
+__host__ __device__ constexpr int ts_chan_bytes(int W)
+{
+    return W * (4 * ((128 + (W / 4 - 1) - 2) / (W / 4 - 1) + 1) + 8);
+}
 
 // (environment, output row, column) of a pixel that advances by a fixed number of pixels per step
 struct PixelWalk {
@@ -290,15 +296,20 @@ __device__ __forceinline__ void ts_rows(const Conv1Plan& pl, int n, int e0, int 
     nB = rows - nA;
 }
 
+// WC: the frame width when it is known at compile time (the converter's 32 loads per row then use
+// immediate offsets instead of computed pointers; its warps are bound by instruction issue), 0 = any.
+template <int WC>
 __global__ void __launch_bounds__(kTsThreads, 2)
 conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
 {
     const Conv1Plan& pl = p.pl;
+    const int W = WC ? WC : pl.W;
+    const int chan_bytes = WC ? ts_chan_bytes(WC) : pl.ts_chan_bytes;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t w_bar, u8_full[kTsStagesMax], u8_empty[kTsStagesMax], q_full[4], q_empty[4], d_full[2], d_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float s_bias[32];
+    __shared__ __align__(16) float s_bias[32];
     volatile int* abortp = &abort_flag;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -341,15 +352,15 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 if (!mbar_wait(&u8_empty[s], (((uint32_t)(it / NU)) & 1u) ^ 1u, abortp, p.status, 31)) break;
                 int nA, nB;
                 ts_rows(pl, p.n, first.e, first.y, first.x, nA, nB);
-                const uint32_t bytesA = (uint32_t)((4 * nA + 4) * pl.W), bytesB = nB ? (uint32_t)((4 * nB + 4) * pl.W) : 0u;
+                const uint32_t bytesA = (uint32_t)((4 * nA + 4) * W), bytesB = nB ? (uint32_t)((4 * nB + 4) * W) : 0u;
                 mbar_arrive_expect_tx(&u8_full[s], (bytesA + bytesB) * pl.C);
                 // staged layout: channel c at c * ts_chan_bytes; inside it the rows of e0, then the rows of e0 + 1
                 uint8_t* dst = s_u8 + s * pl.ts_stage_bytes;
-                const uint8_t* srcA = p.obs + (size_t)first.e * frame + (size_t)(4 * first.y) * pl.W;
-                for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * pl.ts_chan_bytes, srcA + c * chan, bytesA, &u8_full[s]);
+                const uint8_t* srcA = p.obs + (size_t)first.e * frame + (size_t)(4 * first.y) * W;
+                for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * chan_bytes, srcA + c * chan, bytesA, &u8_full[s]);
                 if (nB) {
                     const uint8_t* srcB = p.obs + (size_t)(first.e + 1) * frame;
-                    for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * pl.ts_chan_bytes + bytesA, srcB + c * chan, bytesB, &u8_full[s]);
+                    for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * chan_bytes + bytesA, srcB + c * chan, bytesB, &u8_full[s]);
                 }
             }
         }
@@ -389,26 +400,23 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         int it = 0;
         for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, first.advance(pl.H1, pl.W1), mine.advance(pl.H1, pl.W1)) {
             const int s = it % NU;
-            const bool valid = mine.e < p.n;
             // Staged input row under this pixel's window: four rows per output row since the tile's
-            // first one, plus the four extra rows that close the first environment's part.
+            // first one, plus the four extra rows that close the first environment's part.  Rows past
+            // the end of the batch read the start of the buffer: their results are never stored.
             const int segB = mine.e != first.e;
             const int row = 4 * ((segB ? pl.H1 : 0) + mine.y - first.y + segB + h);
+            const int off = mine.e < p.n ? row * W + 4 * mine.x : 0;
             if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 35)) break;
-            const uint8_t* src = s_u8 + s * pl.ts_stage_bytes + row * pl.W + 4 * mine.x;
+            const uint8_t* src = s_u8 + s * pl.ts_stage_bytes + off;
             bool alive = true;
 #pragma unroll
             for (int dx = 0; dx < 2; ++dx) {
                 uint32_t r[32];
-                const uint8_t* pc = src + 4 * dx;
 #pragma unroll
-                for (int c = 0; c < 4; ++c, pc += pl.ts_chan_bytes) {
-                    const uint8_t* pr = pc;
+                for (int c = 0; c < 4; ++c) {
 #pragma unroll
-                    for (int uy = 0; uy < 4; ++uy, pr += pl.W) {
-                        const uint32_t w = valid ? *reinterpret_cast<const uint32_t*>(pr) : 0u;
-                        u8x4_to_h4(w, r[c * 8 + uy * 2], r[c * 8 + uy * 2 + 1]);
-                    }
+                    for (int uy = 0; uy < 4; ++uy)
+                        u8x4_to_h4(*reinterpret_cast<const uint32_t*>(src + c * chan_bytes + uy * W + 4 * dx), r[c * 8 + uy * 2], r[c * 8 + uy * 2 + 1]);
                 }
                 if (dx == 1) mbar_arrive(&u8_empty[s]);       // the staged rows are in registers
                 if (!mbar_wait_warp(&q_empty[2 * h + dx], ((uint32_t)it & 1u) ^ 1u, abortp, p.status, 36)) { alive = false; break; }
@@ -447,13 +455,17 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 if (mine.e < p.n) {
                     uint32_t pk[8];
 #pragma unroll
-                    for (int hh = 0; hh < 8; ++hh) {
+                    for (int hh = 0; hh < 8; hh += 2) {
                         const int c = 2 * hh;
-                        const float a0 = __uint_as_float(v0[c]) + __uint_as_float(v1[c]);
-                        const float a1 = __uint_as_float(v0[c + 1]) + __uint_as_float(v1[c + 1]);
-                        __half2 tt = __floats2half2_rn(fmaf(a0, inv, s_bias[j + c]), fmaf(a1, inv, s_bias[j + c + 1]));
-                        tt = __hmin2(__hmax2(tt, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
-                        pk[hh] = *reinterpret_cast<uint32_t*>(&tt);
+                        const float4 b4 = *reinterpret_cast<const float4*>(&s_bias[j + c]);
+                        __half2 t0 = __floats2half2_rn(fmaf(__uint_as_float(v0[c]) + __uint_as_float(v1[c]), inv, b4.x),
+                                                       fmaf(__uint_as_float(v0[c + 1]) + __uint_as_float(v1[c + 1]), inv, b4.y));
+                        __half2 t1 = __floats2half2_rn(fmaf(__uint_as_float(v0[c + 2]) + __uint_as_float(v1[c + 2]), inv, b4.z),
+                                                       fmaf(__uint_as_float(v0[c + 3]) + __uint_as_float(v1[c + 3]), inv, b4.w));
+                        t0 = __hmin2(__hmax2(t0, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
+                        t1 = __hmin2(__hmax2(t1, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
+                        pk[hh] = *reinterpret_cast<uint32_t*>(&t0);
+                        pk[hh + 1] = *reinterpret_cast<uint32_t*>(&t1);
                     }
                     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                                  ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
@@ -513,8 +525,7 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     // (a tile then touches at most two environments)
     pl->ts = pl->cpt == 1 && pl->H1 * pl->W1 >= 128;
     if (pl->ts) {
-        const int max_rows = (128 + pl->W1 - 2) / pl->W1 + 1;             // output rows one tile can touch
-        pl->ts_chan_bytes = g.W * (4 * max_rows + 8);                     // one channel of a staged tile (a multiple of 16)
+        pl->ts_chan_bytes = ts_chan_bytes(g.W);                           // one channel of a staged tile (a multiple of 16)
         pl->ts_stage_bytes = (g.C * pl->ts_chan_bytes + 127) / 128 * 128;
         int st = (100 * 1024 - 4 * kChunkBytes) / pl->ts_stage_bytes;     // two CTAs per SM
         if (st > kTsStagesMax) st = kTsStagesMax;
@@ -557,8 +568,10 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
     if (pl.ts && (long)n * pl.H1 * pl.W1 < (1L << 31) - 128 * 2 * sm_count) {
         static int ts_smem_set = 0;
         if (ts_smem_set < pl.ts_smem_bytes) {
-            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.ts_smem_bytes));
-            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<84>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.ts_smem_bytes));
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<84>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.ts_smem_bytes));
+            HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<0>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
             ts_smem_set = pl.ts_smem_bytes;
         }
         const long total_px = (long)n * pl.H1 * pl.W1;
@@ -566,7 +579,8 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
         int grid = 2 * sm_count;
         if (grid > tiles) grid = tiles;
         Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
-        HTS_CUDA(launch_pdl(conv1_ts_kernel, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
+        if (pl.W == 84) HTS_CUDA(launch_pdl(conv1_ts_kernel<84>, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
+        else HTS_CUDA(launch_pdl(conv1_ts_kernel<0>, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
         note_launch();
         return HTS_OK;
     }
