@@ -31,9 +31,9 @@ if ROOT not in sys.path:
 import hts_workloads as wl  # noqa: E402
 
 WORKLOAD = 3                       # hts_workloads.CONFIGS index
-# dram__bytes_read.sum + dram__bytes_write.sum of one conv1_tc_kernel<1> launch at this workload (n = 1024),
+# dram__bytes_read.sum + dram__bytes_write.sum of one conv1_ts_kernel<84> launch at this workload (n = 1024),
 # from the ncu capture summarised in profiles/actor_step_cfg3_n1024.md; reported only for that kernel
-CONV1_DRAM_TRAFFIC_BYTES = 28954880 + 39936
+CONV1_DRAM_TRAFFIC_BYTES = 28958464 + 141312
 METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
 UNIT = "env-steps/s"
 SEED = 0x5EED
@@ -76,7 +76,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
             self.proc = None
@@ -432,7 +432,7 @@ def run_ours(args) -> None:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
