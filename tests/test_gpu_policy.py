@@ -105,6 +105,31 @@ def test_ragged_batch_sizes(n):
         pol.close()
 
 
+@pytest.mark.parametrize("C,H,W,n", [(4, 64, 96, 77),     # 4 channels, width not 84: generic-width tensor-memory conv1; FC split 8
+                                     (8, 84, 84, 33),     # 8 channels: shared-memory conv1 with two planes per tap
+                                     (4, 36, 44, 150),    # image smaller than one 128-pixel tile: shared-memory conv1
+                                     (4, 100, 84, 41)])   # tiles straddle environments at other offsets (24 x 20 outputs)
+def test_other_frame_shapes(C, H, W, n):
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS[2], C=C, H=H, W=W)
+    pol = Policy(cfg, max_batch=n)
+    try:
+        obs = wl.make_obs(cfg, n, batch_index=H + W)
+        ids = np.arange(500, 500 + n, dtype=np.int32)
+        got = pol.step(obs, ids, 2, 4242)
+        rows = np.arange(n) if n <= 40 else np.sort(np.random.default_rng(n).choice(n, 40, replace=False))
+        wt = orc.Weights(pol.params)
+        ref = orc.policy_step(wt, obs[rows], ids[rows], 2, 4242)
+        check_against_oracle(cfg, {k: v[rows] for k, v in got.items()}, ref, TOL["bf16"])
+        taps = orc.policy_forward(wt, obs[rows[:4]], taps=True)
+        m = int(rows[3]) + 1
+        for layer, name in ((1, "conv1"), (2, "conv2"), (3, "conv3")):
+            err = rel_err(pol.activation(layer, m)[rows[:4]], taps[name])
+            assert err <= TOL["bf16"], (name, err)
+    finally:
+        pol.close()
+
+
 def test_uniform_stream_is_bit_exact():
     n, A, seed = 777, 19, 0xFEDCBA9876543210
     g = np.random.default_rng(0)
