@@ -11,9 +11,10 @@
 // A CTA is a pipeline of four roles over its units: one thread issues bulk copies
 // (cp.async.bulk, one per channel) of the band's uint8 rows into a ring of staged bands; eight
 // warps turn a staged band into fp16 (a zero-extended byte is the fp16 subnormal b * 2^-24, exact;
-// 2^24 / 255 is folded into the accumulator scale) and write a ring of 64-channel planes (three or four); one thread issues 16 * planes
-// tcgen05.mma (128 x 32 x 16) into one of two accumulators in tensor memory; four more warps read
-// an accumulator back, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
+// 2^24 / 255 is folded into the accumulator scale) and write a ring of 64-channel planes (three or
+// four); two threads issue the tcgen05.mma (128 x 32 x 16), thread h the 8 * planes of filter row
+// dy = h into its own accumulator in tensor memory; four more warps read the two accumulators
+// back, add them, apply scale, bias and ReLU and store fp16 in the layout conv2 reads.
 // Wide inputs (many planes) fall back to one tile buffer and two staged bands to fit.
 #include "conv1_tc.cuh"
 #include "tc_ptx.cuh"
@@ -23,7 +24,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 448;                   // warp 0 copies, warp 1 MMA issue, warps 2..9 convert, warps 10..13 epilogue
+constexpr int kThreads = 480;                   // warp 0 copies, warps 1 and 14 MMA issue, warps 2..9 convert, warps 10..13 epilogue
 constexpr int kConverters = 256;
 constexpr int kMaxPlanes = 4;
 constexpr int kMaxU8 = 6;
@@ -79,14 +80,14 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
         for (int s = 0; s < kMaxU8; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], kConverters); }
-        for (int s = 0; s < kMaxPlanes; ++s) { mbar_init(&plane_full[s], kConverters); mbar_init(&plane_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], kWorkers); }
+        for (int s = 0; s < kMaxPlanes; ++s) { mbar_init(&plane_full[s], kConverters); mbar_init(&plane_empty[s], 2); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 2); mbar_init(&d_empty[s], kWorkers); }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmW);
     }
     if (threadIdx.x >= 64 && threadIdx.x < 96) s_bias[threadIdx.x - 64] = p.bias[threadIdx.x - 64];
-    if (warp == 1) tmem_alloc(&tmem_slot, 64);
+    if (warp == 1) tmem_alloc(&tmem_slot, 128);           // two buffers x two accumulators (dy = 0, 1) x 32 columns
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -114,9 +115,11 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                     bulk_load(dst + c * band_in_rows * pl.W, src + (size_t)c * pl.H * pl.W, bytes, &u8_full[s]);
             }
         }
-    } else if (warp == 1) {
-        // ---- MMA issue
+    } else if (warp == 1 || warp == 14) {
+        // ---- MMA issue: thread h takes the two taps of filter row dy = h of every plane into its own
+        //      accumulator (one thread issues an MMA every 60 to 130 clocks, the tensor core needs 40)
         if (lane == 0) {
+            const int h = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc = instr_desc_f16(0, 128, 32);
             bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 12);
             int it = 0, pb = 0;
@@ -124,6 +127,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
             for (int u = blockIdx.x; alive && u < units; u += gridDim.x, ++it) {
                 const int db = it & 1;
                 if (!mbar_wait(&d_empty[db], (((uint32_t)it >> 1) & 1u) ^ 1u, abortp, p.status, 16)) break;
+                const uint32_t d_addr = tmem_d + db * 64 + h * 32;
                 uint32_t acc = 0;
 #pragma unroll
                 for (int pln = 0; pln < CPT; ++pln) {     // planes arrive one by one: MMAs of plane k overlap the conversion of k+1
@@ -131,12 +135,13 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                     tc_fence_after();
                     const uint32_t p_addr = a_tile + pb * plane_bytes;
 #pragma unroll
-                    for (int tap = 0; tap < 4; ++tap) {
-                        const int shift = (tap >> 1) * pl.Ws + (tap & 1);
+                    for (int dx = 0; dx < 2; ++dx) {
+                        const int tap = 2 * h + dx;
+                        const int shift = h * pl.Ws + dx;
                         const uint64_t adesc = smem_desc_sw128(p_addr + shift * 128);
                         const uint64_t bdesc = smem_desc_sw128(a_w + (tap * CPT + pln) * kChunkBytes);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) { mma_f16_ss(tmem_d + db * 32, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
+                        for (int k = 0; k < 4; ++k) { mma_f16_ss(d_addr, adesc + 2 * k, bdesc + 2 * k, idesc, acc); acc = 1; }
                     }
                     mma_commit(&plane_empty[pb]);
                     if (++pb == NP) { pb = 0; pph ^= 1u; }
@@ -187,8 +192,8 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
             }
             if (alive) mbar_arrive(&u8_empty[s]);
         }
-    } else {
-        // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1
+    } else if (warp < 14) {
+        // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1 and add the two accumulators
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const float inv = *p.inv_scale;
@@ -200,25 +205,31 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
             const int y0 = band * pl.R;
             if (!mbar_wait_warp(&d_full[db], ((uint32_t)it >> 1) & 1u, abortp, p.status, 15)) break;
             tc_fence_after();
-            uint32_t v[32];
-            tmem_ld_32x32(tmem_d + db * 32 + ((uint32_t)(q * 32) << 16), v);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(&d_empty[db]);
+            const uint32_t taddr = tmem_d + db * 64 + ((uint32_t)(q * 32) << 16);
             const int yy = y0 + ey;
-            if (ey < pl.R && yy < pl.H1 && ex < pl.W1) {
-                __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (ex >> 1)) * 128 +
-                              ((yy & 1) * 2 + (ex & 1)) * 32;
+            const bool valid = ey < pl.R && yy < pl.H1 && ex < pl.W1;
+            __half* dst = p.out + ((size_t)env * pl.P1s + (size_t)(yy >> 1) * pl.W1s + (ex >> 1)) * 128 +
+                          ((yy & 1) * 2 + (ex & 1)) * 32;
 #pragma unroll
-                for (int j = 0; j < 32; j += 16) {
+            for (int j = 0; j < 32; j += 16) {
+                uint32_t v0[16], v1[16];
+                tmem_ld_32x16(taddr + j, v0);               // dy = 0 taps
+                tmem_ld_32x16(taddr + 32 + j, v1);          // dy = 1 taps
+                tmem_ld_wait();
+                if (j == 16) {
+                    tc_fence_before();
+                    mbar_arrive(&d_empty[db]);
+                }
+                if (valid) {
                     uint32_t pk[8];
 #pragma unroll
-                    for (int h = 0; h < 8; ++h) {
-                        const int c = j + 2 * h;
-                        __half2 t = __floats2half2_rn(fmaf(__uint_as_float(v[c]), inv, s_bias[c]),
-                                                      fmaf(__uint_as_float(v[c + 1]), inv, s_bias[c + 1]));
+                    for (int hh = 0; hh < 8; ++hh) {
+                        const int c = 2 * hh;
+                        const float a0 = __uint_as_float(v0[c]) + __uint_as_float(v1[c]);
+                        const float a1 = __uint_as_float(v0[c + 1]) + __uint_as_float(v1[c + 1]);
+                        __half2 t = __floats2half2_rn(fmaf(a0, inv, s_bias[j + c]), fmaf(a1, inv, s_bias[j + c + 1]));
                         t = __hmin2(__hmax2(t, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
-                        pk[h] = *reinterpret_cast<uint32_t*>(&t);
+                        pk[hh] = *reinterpret_cast<uint32_t*>(&t);
                     }
                     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                                  ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
@@ -233,7 +244,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_d, 64);
+    if (warp == 1) tmem_dealloc(tmem_d, 128);
 }
 
 // ---------------------------------------------------------------------------------------------
