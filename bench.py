@@ -173,6 +173,40 @@ def run_ncu_case(steps: int) -> None:
 
 
 # ------------------------------------------------------------------------------------------------
+def run_batch_sweep() -> None:
+    """Actor-step time against the executor batch size, 1..8192 rows of the 8192-environment pool of the
+    asynchronous-executor configuration (4x84x84 frames, 18 actions); prints a markdown table."""
+    import torch
+    import paper_2012_09849_b200 as hts
+    cfg = wl.CONFIGS[5]
+    pool = cfg.N
+    ctx = hts.hts_policy_create(cfg.C, cfg.H, cfg.W, cfg.A, hts.HTS_DTYPE_BF16, pool)
+    hts.hts_policy_load_weights(ctx, hts.weights_to_device(wl.make_weights(cfg), hts.HTS_DTYPE_BF16))
+    obs = [torch.from_numpy(wl.make_obs(cfg, pool, batch_index=i)).cuda() for i in range(2)]
+    ids = torch.arange(pool, dtype=torch.int32, device="cuda")
+    act = torch.empty(pool, dtype=torch.int32, device="cuda")
+    f = [torch.empty(pool, device="cuda") for _ in range(3)]
+    macs = macs_per_env_step(cfg)
+    print("| batch n | us per step | env-steps/s | TFLOP/s |")
+    print("|---|---|---|---|")
+    n = 1
+    while n <= pool:
+        reps = 50 if n <= 1024 else 20
+        for t in range(5):
+            hts.hts_policy_step(ctx, obs[t % 2], ids, None, t, SEED, n, act, *f)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for t in range(reps):
+            hts.hts_policy_step(ctx, obs[t % 2], ids, None, t, SEED, n, act, *f)
+        b.record(); torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(b) / reps
+        print(f"| {n} | {us:.1f} | {n / us * 1e6:.3g} | {2 * macs * n / us / 1e6:.1f} |", flush=True)
+        n *= 2
+    hts.hts_policy_destroy(ctx)
+
+
+# ------------------------------------------------------------------------------------------------
 def run_ours(args) -> None:
     import torch
     import paper_2012_09849_b200 as hts
@@ -327,6 +361,25 @@ def run_ours(args) -> None:
                 "us_per_launch": top_us}
     whole_tf = 2.0 * macs_per_env_step(cfg) * value / world / 1e12
 
+    # ---- the executor-facing form: frames gathered by slot from a state buffer (one ring entry), outputs
+    #      scattered to the same slots of a storage row; slots = a random permutation of the pool
+    perm = torch.from_numpy(np.random.default_rng(SEED).permutation(N).astype(np.int32)).to(dev)
+    p_perm = perm.data_ptr()
+    st0 = store[0]
+
+    def indexed_steps(count):
+        for t in range(count):
+            hts.hts_policy_step_indexed(ctx, p_obs[t % ring], N, p_perm, p_ids, None, t % T, SEED, N,
+                                        st0.p_act[t % T], st0.p_logp[t % T], st0.p_val[t % T], st0.p_ent[t % T],
+                                        h_act_stream)
+    indexed_steps(8)
+    torch.cuda.synchronize()
+    i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    i0.record(s_act)
+    indexed_steps(2 * T)
+    i1.record(s_act); torch.cuda.synchronize()
+    indexed_us = 1e3 * i0.elapsed_time(i1) / (2 * T)
+
     # ---- end to end through the host-buffer entry points
     if rank == 0 or dist is not None:
         h_act = torch.empty(T, N, dtype=torch.int32).pin_memory()
@@ -421,6 +474,7 @@ def run_ours(args) -> None:
                 "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
                          "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
         "actor_step_us": 1e3 * ms / (args.steps * T),
+        "indexed_actor_step_us": indexed_us,
         "large_batch_actor_step": big,
         "cpu_baseline": cpu,
     }
@@ -439,8 +493,12 @@ def main():
     ap.add_argument("--ncu-case", type=int, default=0, metavar="STEPS",
                     help="profiling driver: run STEPS actor steps of the bench workload plus one GAE and exit "
                          "(no timing; for use under ncu)")
+    ap.add_argument("--batch-sweep", action="store_true",
+                    help="print actor-step time against the batch size (1..8192) and exit")
     args = ap.parse_args()
-    if args.ncu_case > 0:
+    if args.batch_sweep:
+        run_batch_sweep()
+    elif args.ncu_case > 0:
         run_ncu_case(args.ncu_case)
     elif args.impl == "reference":
         run_reference(args)

@@ -107,6 +107,30 @@ hts_status hts_policy_step(hts_ctx *ctx, const uint8_t *obs, const int32_t *env_
                            int32_t *actions, float *logp, float *values, float *entropy,
                            float *logits_or_null, void *cuda_stream);
 
+/* The executor-facing form of the same step (Section 4.1: executors write states
+ * to the state buffer, actors read from it, and their outputs go to the data
+ * storage used by the learner): the frames of the batch are gathered from a
+ * device-resident state buffer by slot, and each row's outputs are scattered to
+ * the same slot of one row of the [T, pool] rollout storage, with no copy in
+ * between.  A batch is any subset of the pool in any order (the executor batches
+ * of an asynchronous step).
+ *   state_buffer  DEVICE u8  [pool,C,H,W]  one frame per environment slot
+ *   slots         DEVICE i32 [n]           slot of each row, each in [0, pool)
+ *   env_ids, t_per_env, t, seed, n         as in hts_policy_step (env_ids feed the
+ *                                          random stream; they need not equal slots)
+ *   actions_row, logp_row, values_row, entropy_row
+ *                 DEVICE [pool]  out       row t of the storage; only the entries
+ *                                          at the n slots are written
+ * Outputs equal, bit for bit, those of hts_policy_step on the gathered frames.
+ * If two rows name the same slot, one of them is kept.  A slot outside [0, pool)
+ * is not dereferenced: that row writes nothing and hts_last_async_error reports
+ * INVALID_ARG.  Errors otherwise as hts_policy_step.                            */
+hts_status hts_policy_step_indexed(hts_ctx *ctx, const uint8_t *state_buffer, int32_t pool,
+                                   const int32_t *slots, const int32_t *env_ids,
+                                   const int32_t *t_per_env, int32_t t, uint64_t seed, int32_t n,
+                                   int32_t *actions_row, float *logp_row, float *values_row,
+                                   float *entropy_row, void *cuda_stream);
+
 /* Same operation with HOST buffers: copies obs/env_ids/t_per_env to the device,
  * runs the step, copies the four outputs (and logits if asked) back and waits for
  * them.  Uses staging buffers owned by the context (allocated at create time).
@@ -142,8 +166,9 @@ hts_status hts_policy_profile(hts_ctx *ctx, int32_t enable);
 hts_status hts_policy_profile_read(hts_ctx *ctx, int32_t kernel, float *total_ms, int32_t *launches);
 const char *hts_policy_kernel_name(int32_t kernel);
 
-/* Reads and clears the device status word of the context (set by a bounded wait
- * that ran out).  Synchronises with the device.  HTS_OK if nothing was recorded.  */
+/* Reads and clears the device status word of the context: HTS_ERR_TIMEOUT if a
+ * bounded wait ran out, HTS_ERR_INVALID_ARG if hts_policy_step_indexed met a slot
+ * outside the pool, HTS_OK if nothing was recorded.  Synchronises with the device. */
 hts_status hts_last_async_error(hts_ctx *ctx);
 
 void hts_policy_destroy(hts_ctx *ctx);

@@ -22,7 +22,7 @@ STATUS_NAMES = ["HTS_OK", "HTS_ERR_INVALID_ARG", "HTS_ERR_SHAPE", "HTS_ERR_ALLOC
                 "HTS_ERR_TIMEOUT", "HTS_ERR_UNSUPPORTED"]
 WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
                 "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
-EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_host",
+EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_indexed", "hts_policy_step_host",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
            "hts_gae_host", "hts_policy_step_noalloc", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
@@ -66,6 +66,7 @@ def lib():
         step = [vp, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp, vp, vp]
         L.hts_policy_step.argtypes = step
         L.hts_policy_step_host.argtypes = step
+        L.hts_policy_step_indexed.argtypes = [vp, vp, i32, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp, vp]
         L.hts_policy_read_activation.argtypes = [vp, i32, i32, vp, vp]
         L.hts_action_uniforms.argtypes = [vp, vp, i32, u64, i32, i32, vp, vp]
         L.hts_policy_profile.argtypes = [vp, i32]
@@ -86,7 +87,7 @@ def lib():
         L.hts_last_cuda_error.restype = C.c_char_p
         L.hts_status_string.restype = C.c_char_p
         L.hts_status_string.argtypes = [C.c_int]
-        for name in ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_host",
+        for name in ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_indexed", "hts_policy_step_host",
                      "hts_policy_read_activation", "hts_action_uniforms", "hts_last_async_error", "hts_gae",
                      "hts_gae_host"):
             getattr(L, name).restype = C.c_int
@@ -138,6 +139,13 @@ def hts_policy_step(ctx, obs, env_ids, t_per_env, t, seed, n, actions, logp, val
     _check(lib().hts_policy_step(ctx, _ptr(obs), _ptr(env_ids), _ptr(t_per_env), int(t), int(seed), int(n),
                                  _ptr(actions), _ptr(logp), _ptr(values), _ptr(entropy), _ptr(logits),
                                  _stream(stream)), "hts_policy_step")
+
+
+def hts_policy_step_indexed(ctx, state_buffer, pool, slots, env_ids, t_per_env, t, seed, n, actions_row, logp_row,
+                            values_row, entropy_row, stream=None) -> None:
+    _check(lib().hts_policy_step_indexed(ctx, _ptr(state_buffer), int(pool), _ptr(slots), _ptr(env_ids), _ptr(t_per_env),
+                                         int(t), int(seed), int(n), _ptr(actions_row), _ptr(logp_row), _ptr(values_row),
+                                         _ptr(entropy_row), _stream(stream)), "hts_policy_step_indexed")
 
 
 def hts_policy_step_host(ctx, obs, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy,

@@ -44,6 +44,16 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 
 inline int conv_out(int extent, int k, int s) { return (extent - k) / s + 1; }
 
+// Executor-facing addressing of a step (state buffer -> actors -> storage row, Section 4.1): row e of the
+// batch reads frame slots[e] of a pool of `pool` frames and writes its outputs at index slots[e].
+// slots == nullptr: frames and outputs are dense, row e at index e.  A slot outside [0, pool) is
+// reported through the device status word (kStatusBadSlot); that row reads frame 0 and writes nothing.
+struct Indexing {
+    const int32_t* slots = nullptr;
+    int pool = 0;
+};
+constexpr int kStatusBadSlot = 100;
+
 // Geometry of the fixed four-layer network for one observation shape.
 struct Geometry {
     int C, H, W, A;
@@ -72,7 +82,7 @@ struct RefWorkspace { float *a1, *a2, *a3, *h; };   // NCHW fp32 activations, [n
 hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& src,
                                const RefWeights& dst, cudaStream_t s);
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
-                       const uint8_t* obs, int n, Profiler& prof, cudaStream_t s);
+                       const uint8_t* obs, const Indexing& ix, int* status, int n, Profiler& prof, cudaStream_t s);
 
 // ---- the tensor-core path (bf16 weights) -------------------------------------------------------
 struct TcState;
@@ -80,9 +90,10 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
                      bool (*alloc)(void* ctx, void** p, size_t bytes), void* alloc_ctx);
 void tc_destroy(TcState* t);
 hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s);
-hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cudaStream_t s);
+hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n, Profiler& prof, cudaStream_t s);
 hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
-                    int32_t* actions, float* logp, float* values, float* entropy, float* logits, cudaStream_t s);
+                    const Indexing& ix, int32_t* actions, float* logp, float* values, float* entropy, float* logits,
+                    cudaStream_t s);
 hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s);
 
 // ---- heads + distribution + sampling epilogue (both paths) --------------------------------
@@ -91,8 +102,8 @@ hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStre
 hts_status launch_heads(const float* h_partials, int num_splits, size_t split_stride,
                         const float* fc_bias, const float* whead, const float* bhead, int A,
                         const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
-                        uint64_t seed, int n, int32_t* actions, float* logp, float* values,
-                        float* entropy, float* logits, float* h_out, cudaStream_t s);
+                        uint64_t seed, int n, const Indexing& ix, int* status, int32_t* actions, float* logp,
+                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s);
 
 hts_status launch_uniforms(const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed, int n,
                            int A, float* out, cudaStream_t s);

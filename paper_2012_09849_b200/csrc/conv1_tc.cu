@@ -34,12 +34,24 @@ constexpr int kChunkBytes = 32 * 64 * 2;        // one weight K chunk: 32 rows x
 struct Conv1Params {
     Conv1Plan pl;
     const uint8_t* obs;
+    const int32_t* slots;   // frame of each row in obs, or nullptr: row e is frame e
+    int pool;               // frames in obs when slots are given
     int n;
     const float* bias;
     const float* inv_scale;
     __half* out;
     int* status;
 };
+
+// Frame index of batch row e: e itself, or its slot in the pool.  A slot outside the pool is
+// recorded in the status word and frame 0 is read instead (the heads kernel drops that row).
+__device__ __forceinline__ size_t frame_of(const Conv1Params& p, int e)
+{
+    if (!p.slots) return (size_t)e;
+    const int sl = p.slots[e];
+    if ((unsigned)sl >= (unsigned)p.pool) { atomicCAS(p.status, 0, kStatusBadSlot); return 0; }
+    return (size_t)sl;
+}
 
 // Four bytes -> four fp16 values without arithmetic: a byte b zero-extended to 16 bits is the fp16
 // subnormal b * 2^-24, which the tensor core multiplies exactly; the 2^24 goes into the accumulator scale.
@@ -109,7 +121,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 int rows = pl.H - r0; rows = rows > band_in_rows ? band_in_rows : rows;
                 const uint32_t bytes = (uint32_t)(rows * pl.W);
                 mbar_arrive_expect_tx(&u8_full[s], bytes * pl.C);
-                const uint8_t* src = p.obs + ((size_t)env * pl.C * pl.H + r0) * pl.W;
+                const uint8_t* src = p.obs + (frame_of(p, env) * pl.C * pl.H + r0) * pl.W;
                 uint8_t* dst = s_u8 + s * pl.u8_stage_bytes;
                 for (int c = 0; c < pl.C; ++c)
                     bulk_load(dst + c * band_in_rows * pl.W, src + (size_t)c * pl.H * pl.W, bytes, &u8_full[s]);
@@ -367,10 +379,10 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 mbar_arrive_expect_tx(&u8_full[s], (bytesA + bytesB) * pl.C);
                 // staged layout: channel c at c * ts_chan_bytes; inside it the rows of e0, then the rows of e0 + 1
                 uint8_t* dst = s_u8 + s * pl.ts_stage_bytes;
-                const uint8_t* srcA = p.obs + (size_t)first.e * frame + (size_t)(4 * first.y) * W;
+                const uint8_t* srcA = p.obs + frame_of(p, first.e) * frame + (size_t)(4 * first.y) * W;
                 for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * chan_bytes, srcA + c * chan, bytesA, &u8_full[s]);
                 if (nB) {
-                    const uint8_t* srcB = p.obs + (size_t)(first.e + 1) * frame;
+                    const uint8_t* srcB = p.obs + frame_of(p, first.e + 1) * frame;
                     for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * chan_bytes + bytesA, srcB + c * chan, bytesB, &u8_full[s]);
                 }
             }
@@ -556,7 +568,7 @@ hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __ha
     return HTS_OK;
 }
 
-hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, int n,
+hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, const Indexing& ix, int n,
                         const float* bias, const float* inv_scale, __half* out, int* status, cudaStream_t s)
 {
     static int sm_count = 0, max_smem_set = 0;
@@ -589,7 +601,7 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
         const int tiles = (int)((total_px + 127) / 128);
         int grid = 2 * sm_count;
         if (grid > tiles) grid = tiles;
-        Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
+        Conv1Params p{pl, obs, ix.slots, ix.pool, n, bias, inv_scale, out, status};
         if (pl.W == 84) HTS_CUDA(launch_pdl(conv1_ts_kernel<84>, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
         else HTS_CUDA(launch_pdl(conv1_ts_kernel<0>, dim3(grid), dim3(kTsThreads), (size_t)pl.ts_smem_bytes, s, weight_map, p));
         note_launch();
@@ -599,7 +611,7 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
     const int units = n * pl.bands;
     int grid = sm_count * (per_sm < 1 ? 1 : per_sm);
     if (grid > units) grid = units;
-    Conv1Params p{pl, obs, n, bias, inv_scale, out, status};
+    Conv1Params p{pl, obs, ix.slots, ix.pool, n, bias, inv_scale, out, status};
     if (pl.cpt == 1) HTS_CUDA(launch_pdl(conv1_tc_kernel<1>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
     else if (pl.cpt == 2) HTS_CUDA(launch_pdl(conv1_tc_kernel<2>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));
     else HTS_CUDA(launch_pdl(conv1_tc_kernel<4>, dim3(grid), dim3(kThreads), (size_t)pl.smem_bytes, s, weight_map, p));

@@ -32,7 +32,8 @@ hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __ha
                               cudaStream_t s);
 
 // out: fp16 rows [env*P1s + (y/2)*W1s + x/2][128], column ((y%2)*2 + x%2)*32 + o
-hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, int n,
+// ix: dense frames (row e = frame e of obs) or frames gathered by slot from a pool (see Indexing)
+hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, const Indexing& ix, int n,
                         const float* bias, const float* inv_scale, __half* out, int* status, cudaStream_t s);
 
 }  // namespace hts

@@ -63,7 +63,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
              const float* __restrict__ fc_bias, const float* __restrict__ whead,
              const float* __restrict__ bhead, int A, const int32_t* __restrict__ env_ids,
              const int32_t* __restrict__ t_per_env, int32_t t_scalar, uint32_t key0, uint32_t key1,
-             int n, int32_t* __restrict__ actions, float* __restrict__ logp,
+             int n, const int32_t* __restrict__ slots, int pool, int* __restrict__ status,
+             int32_t* __restrict__ actions, float* __restrict__ logp,
              float* __restrict__ values, float* __restrict__ entropy, float* __restrict__ logits_out,
              float* __restrict__ h_out)
 {
@@ -163,10 +164,17 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
     }
     if (logits_out) for (int a = lane; a < A; a += 32) logits_out[(size_t)e * A + a] = lg[a];
     if (lane == 0) {
-        actions[e] = best_a;
-        logp[e] = lg[best_a] - lse;
-        values[e] = lg[A];
-        entropy[e] = ent;
+        int o = e;                                       // dense, or the row's slot of the storage row
+        if (slots) {
+            o = slots[e];
+            if ((unsigned)o >= (unsigned)pool) { atomicCAS(status, 0, kStatusBadSlot); o = -1; }
+        }
+        if (o >= 0) {
+            actions[o] = best_a;
+            logp[o] = lg[best_a] - lse;
+            values[o] = lg[A];
+            entropy[o] = ent;
+        }
     }
     __syncwarp();                                      // s_out[wib] is reused by the next environment
     }
@@ -177,8 +185,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
 hts_status launch_heads(const float* h_partials, int num_splits, size_t split_stride,
                         const float* fc_bias, const float* whead, const float* bhead, int A,
                         const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
-                        uint64_t seed, int n, int32_t* actions, float* logp, float* values,
-                        float* entropy, float* logits, float* h_out, cudaStream_t s)
+                        uint64_t seed, int n, const Indexing& ix, int* status, int32_t* actions, float* logp,
+                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s)
 {
     if (num_splits < 1 || num_splits > kMaxSplits) return HTS_ERR_INVALID_ARG;
     const size_t smem = (size_t)(A + 1) * kHidden * sizeof(float);
@@ -201,8 +209,8 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
     int blocks = (n + 7) / 8;
     if (blocks > 2 * sm_count) blocks = 2 * sm_count;
     HTS_CUDA(launch_pdl(heads_kernel, dim3(blocks), dim3(256), smem, s, h_partials, num_splits, split_stride, fc_bias, whead,
-                        bhead, A, env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), n, actions,
-                        logp, values, entropy, logits, h_out));
+                        bhead, A, env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), n, ix.slots,
+                        ix.pool, status, actions, logp, values, entropy, logits, h_out));
     note_launch();
     return HTS_OK;
 }

@@ -88,23 +88,23 @@ hts_status check_step_args(hts_ctx* ctx, const void* obs, const void* env_ids, i
     return HTS_OK;
 }
 
-hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids, const int32_t* t_per_env,
+hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const Indexing& ix, const int32_t* env_ids, const int32_t* t_per_env,
                     int32_t t, uint64_t seed, int32_t n, int32_t* actions, float* logp, float* values,
                     float* entropy, float* logits, cudaStream_t s)
 {
     const Geometry& g = ctx->g;
     hts_status st;
     if (ctx->tc) {
-        st = tc_forward(ctx->tc, obs, n, ctx->prof, s);
+        st = tc_forward(ctx->tc, obs, ix, n, ctx->prof, s);
         if (st != HTS_OK) return st;
         ctx->prof.begin(K_HEADS, s);
-        st = tc_heads(ctx->tc, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy, logits, s);
+        st = tc_heads(ctx->tc, env_ids, t_per_env, t, seed, n, ix, actions, logp, values, entropy, logits, s);
     } else {
-        st = ref_forward(g, ctx->rw, ctx->rws, obs, n, ctx->prof, s);
+        st = ref_forward(g, ctx->rw, ctx->rws, obs, ix, ctx->status, n, ctx->prof, s);
         if (st != HTS_OK) return st;
         ctx->prof.begin(K_HEADS, s);
         st = launch_heads(ctx->rws.h, 1, 0, nullptr, ctx->rw.whead, ctx->rw.bhead, g.A, env_ids, t_per_env, t,
-                          seed, n, actions, logp, values, entropy, logits, nullptr, s);
+                          seed, n, ix, ctx->status, actions, logp, values, entropy, logits, nullptr, s);
     }
     if (st != HTS_OK) return st;
     ctx->prof.end(K_HEADS, s);
@@ -193,8 +193,27 @@ hts_status hts_policy_step(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_
     const Range outr[] = {{actions, nn * 4}, {logp, nn * 4}, {values, nn * 4}, {entropy, nn * 4},
                           {logits_or_null, nn * ctx->g.A * 4}};
     if (any_overlap(in, 3, outr, 5)) return HTS_ERR_INVALID_ARG;
-    return run_step(ctx, obs, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy, logits_or_null,
+    return run_step(ctx, obs, Indexing{}, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy, logits_or_null,
                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+hts_status hts_policy_step_indexed(hts_ctx* ctx, const uint8_t* state_buffer, int32_t pool, const int32_t* slots,
+                                   const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed,
+                                   int32_t n, int32_t* actions_row, float* logp_row, float* values_row,
+                                   float* entropy_row, void* cuda_stream)
+{
+    hts_status st = check_step_args(ctx, state_buffer, env_ids, n, actions_row, logp_row, values_row, entropy_row);
+    if (st != HTS_OK) return st;
+    if (!slots || pool < 1) return HTS_ERR_INVALID_ARG;
+    const size_t nn = (size_t)n, pp = (size_t)pool;
+    const Range in[] = {{state_buffer, pp * ctx->g.C * ctx->g.H * ctx->g.W}, {slots, nn * 4}, {env_ids, nn * 4},
+                        {t_per_env, nn * 4}};
+    const Range outr[] = {{actions_row, pp * 4}, {logp_row, pp * 4}, {values_row, pp * 4}, {entropy_row, pp * 4}};
+    if (any_overlap(in, 4, outr, 4)) return HTS_ERR_INVALID_ARG;
+    Indexing ix;
+    ix.slots = slots; ix.pool = pool;
+    return run_step(ctx, state_buffer, ix, env_ids, t_per_env, t, seed, n, actions_row, logp_row, values_row, entropy_row,
+                    nullptr, static_cast<cudaStream_t>(cuda_stream));
 }
 
 hts_status hts_policy_step_host(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids,
@@ -209,7 +228,7 @@ hts_status hts_policy_step_host(hts_ctx* ctx, const uint8_t* obs, const int32_t*
     HTS_CUDA(cudaMemcpyAsync(ctx->s_obs, obs, nn * ctx->g.C * ctx->g.H * ctx->g.W, cudaMemcpyHostToDevice, s));
     HTS_CUDA(cudaMemcpyAsync(ctx->s_ids, env_ids, nn * 4, cudaMemcpyHostToDevice, s));
     if (t_per_env) HTS_CUDA(cudaMemcpyAsync(ctx->s_t, t_per_env, nn * 4, cudaMemcpyHostToDevice, s));
-    st = run_step(ctx, ctx->s_obs, ctx->s_ids, t_per_env ? ctx->s_t : nullptr, t, seed, n, ctx->s_act,
+    st = run_step(ctx, ctx->s_obs, Indexing{}, ctx->s_ids, t_per_env ? ctx->s_t : nullptr, t, seed, n, ctx->s_act,
                   ctx->s_logp, ctx->s_val, ctx->s_ent, logits_or_null ? ctx->s_logits : nullptr, s);
     if (st != HTS_OK) return st;
     HTS_CUDA(cudaMemcpyAsync(actions, ctx->s_act, nn * 4, cudaMemcpyDeviceToHost, s));
@@ -250,7 +269,7 @@ hts_status hts_last_async_error(hts_ctx* ctx)
     HTS_CUDA(cudaMemcpy(&word, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word != 0) {
         HTS_CUDA(cudaMemset(ctx->status, 0, sizeof(int)));
-        return HTS_ERR_TIMEOUT;
+        return word == kStatusBadSlot ? HTS_ERR_INVALID_ARG : HTS_ERR_TIMEOUT;
     }
     return HTS_OK;
 }

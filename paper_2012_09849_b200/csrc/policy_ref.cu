@@ -19,7 +19,7 @@ template <typename TIn>
 __global__ void conv_direct_kernel(const TIn* __restrict__ x, const float* __restrict__ w,
                                    const float* __restrict__ b, float* __restrict__ y,
                                    int n, int C, int H, int W, int O, int k, int s, int Ho, int Wo,
-                                   float in_scale)
+                                   float in_scale, const int32_t* __restrict__ slots, int pool, int* __restrict__ status)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t total = (size_t)n * O * Ho * Wo;
@@ -28,7 +28,13 @@ __global__ void conv_direct_kernel(const TIn* __restrict__ x, const float* __res
     const int i = (int)((idx / Wo) % Ho);
     const int o = (int)((idx / ((size_t)Wo * Ho)) % O);
     const size_t e = idx / ((size_t)Wo * Ho * O);
-    const TIn* xe = x + e * (size_t)C * H * W;
+    size_t frame = e;                                   // dense, or the row's frame of the state buffer
+    if (slots) {
+        const int sl = slots[e];
+        if ((unsigned)sl >= (unsigned)pool) { atomicCAS(status, 0, kStatusBadSlot); frame = 0; }
+        else frame = (size_t)sl;
+    }
+    const TIn* xe = x + frame * (size_t)C * H * W;
     const float* wo = w + (size_t)o * C * k * k;
     float acc = 0.f;
     for (int c = 0; c < C; ++c)
@@ -83,22 +89,22 @@ hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& 
 }
 
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
-                       const uint8_t* obs, int n, Profiler& prof, cudaStream_t s)
+                       const uint8_t* obs, const Indexing& ix, int* status, int n, Profiler& prof, cudaStream_t s)
 {
     const int th = 256;
     prof.begin(K_CONV1, s);
     conv_direct_kernel<uint8_t><<<blocks_for((size_t)n * 32 * g.H1 * g.W1, th), th, 0, s>>>(
-        obs, w.w1, w.b1, ws.a1, n, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, 1.0f / 255.0f);
+        obs, w.w1, w.b1, ws.a1, n, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, 1.0f / 255.0f, ix.slots, ix.pool, status);
     HTS_LAUNCH_CHECK("conv1_direct");
     prof.end(K_CONV1, s);
     prof.begin(K_CONV2, s);
     conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H2 * g.W2, th), th, 0, s>>>(
-        ws.a1, w.w2, w.b2, ws.a2, n, 32, g.H1, g.W1, 64, 4, 2, g.H2, g.W2, 1.0f);
+        ws.a1, w.w2, w.b2, ws.a2, n, 32, g.H1, g.W1, 64, 4, 2, g.H2, g.W2, 1.0f, nullptr, 0, nullptr);
     HTS_LAUNCH_CHECK("conv2_direct");
     prof.end(K_CONV2, s);
     prof.begin(K_CONV3, s);
     conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H3 * g.W3, th), th, 0, s>>>(
-        ws.a2, w.w3, w.b3, ws.a3, n, 64, g.H2, g.W2, 64, 3, 1, g.H3, g.W3, 1.0f);
+        ws.a2, w.w3, w.b3, ws.a3, n, 64, g.H2, g.W2, 64, 3, 1, g.H3, g.W3, 1.0f, nullptr, 0, nullptr);
     HTS_LAUNCH_CHECK("conv3_direct");
     prof.end(K_CONV3, s);
     prof.begin(K_FC, s);
@@ -170,8 +176,8 @@ extern "C" hts_status hts_policy_step_noalloc(const hts_net_desc* d, const hts_w
     const RefWeights rw{f(w->conv1_w), f(w->conv1_b), f(w->conv2_w), f(w->conv2_b), f(w->conv3_w), f(w->conv3_b),
                         f(w->fc_w), f(w->fc_b), whead, bhead};
     Profiler off;
-    hts_status st = ref_forward(g, rw, ws, obs, n, off, s);
+    hts_status st = ref_forward(g, rw, ws, obs, Indexing{}, nullptr, n, off, s);
     if (st != HTS_OK) return st;
-    return launch_heads(ws.h, 1, 0, nullptr, whead, bhead, g.A, env_ids, t_per_env, t, seed, n, actions, logp,
-                        values, entropy, logits_or_null, nullptr, s);
+    return launch_heads(ws.h, 1, 0, nullptr, whead, bhead, g.A, env_ids, t_per_env, t, seed, n, Indexing{}, nullptr, actions,
+                        logp, values, entropy, logits_or_null, nullptr, s);
 }

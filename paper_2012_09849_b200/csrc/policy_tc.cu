@@ -382,11 +382,11 @@ hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s)
     return HTS_OK;
 }
 
-hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cudaStream_t s)
+hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n, Profiler& prof, cudaStream_t s)
 {
     const Geometry& g = t->g;
     prof.begin(K_CONV1, s);
-    hts_status st = conv1_launch(t->pl1, t->mW1, obs, n, t->b1, t->inv_scale + L_CONV1, t->a1s, t->status, s);
+    hts_status st = conv1_launch(t->pl1, t->mW1, obs, ix, n, t->b1, t->inv_scale + L_CONV1, t->a1s, t->status, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV1, s);
 
@@ -423,10 +423,11 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, int n, Profiler& prof, cud
 }
 
 hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
-                    int32_t* actions, float* logp, float* values, float* entropy, float* logits, cudaStream_t s)
+                    const Indexing& ix, int32_t* actions, float* logp, float* values, float* entropy, float* logits,
+                    cudaStream_t s)
 {
     return launch_heads(t->hpart, t->splits, (size_t)t->max_batch * 512, t->bfc, t->whead, t->bhead, t->g.A, env_ids,
-                        t_per_env, tt, seed, n, actions, logp, values, entropy, logits, t->h, s);
+                        t_per_env, tt, seed, n, ix, t->status, actions, logp, values, entropy, logits, t->h, s);
 }
 
 hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s)
