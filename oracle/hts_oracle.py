@@ -190,3 +190,35 @@ def gae(rewards, values, dones, bootstrap, gamma: float, lam: float):
     lib().hts_oracle_gae(_p(r), _p(v), _p(d), _p(b), C.c_double(gamma), C.c_double(lam),
                          T, N, _p(adv), _p(ret))
     return adv, ret
+
+
+def evaluate_actions(wt: Weights, obs, actions):
+    """What the learner re-evaluates on stored transitions (Section 3, Eq. 3/4): for each row the
+    log-probability of the action that was taken, the value estimate and the policy entropy (nats).
+    -> dict(logp [n], values [n], entropy [n], logits [n,A])."""
+    actions = np.ascontiguousarray(actions, dtype=np.int64)
+    f = policy_forward(wt, obs)
+    n = actions.shape[0]
+    assert f["logits"].shape[0] == n and np.all((actions >= 0) & (actions < wt.A))
+    logp, ent = np.empty(n), np.empty(n)
+    for e in range(n):
+        lp, h = log_softmax(f["logits"][e])
+        logp[e], ent[e] = lp[actions[e]], h
+    return {"logp": logp, "values": f["value"].copy(), "entropy": ent, "logits": f["logits"]}
+
+
+def a2c_terms(logp, values, entropy, returns):
+    """The three sample means the actor-critic update is built from (Section 3): the policy term of
+    Eq. 4, (1/|D|) sum log pi(a_t|s_t) (R_t - V(s_t)), whose gradient with R_t - V held fixed is Eq. 4's first
+    summand; the value loss J_V = (1/|D|) sum (R_t - V(s_t))^2; and the mean entropy that Eq. 4 weights by alpha.
+    fp64 throughout.  -> (policy_term, value_loss, mean_entropy)."""
+    logp, values, entropy, returns = (np.asarray(a, dtype=np.float64).ravel() for a in (logp, values, entropy, returns))
+    count = logp.size
+    assert count > 0 and values.size == count and entropy.size == count and returns.size == count
+    pol = vl = ent = 0.0
+    for i in range(count):
+        adv = returns[i] - values[i]
+        pol += logp[i] * adv
+        vl += adv * adv
+        ent += entropy[i]
+    return pol / count, vl / count, ent / count

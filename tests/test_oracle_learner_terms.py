@@ -1,0 +1,72 @@
+"""Pins of the oracle's learner-side functions (re-evaluation of stored actions, Eq. 4 sample means)."""
+import os
+
+import numpy as np
+import pytest
+
+import hts_workloads as wl
+from oracle import hts_oracle as orc
+
+GOLD = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "a2c_terms_worked_example.txt")
+
+
+def test_a2c_terms_worked_example():
+    rows, expected = [], None
+    for line in open(GOLD, encoding="utf-8"):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("expected"):
+            expected = [float(x) for x in line.split()[1:]]
+        else:
+            rows.append([float(x) for x in line.split()])
+    a = np.array(rows)
+    got = orc.a2c_terms(a[:, 0], a[:, 1], a[:, 2], a[:, 3])
+    assert list(got) == expected
+
+
+def test_a2c_terms_closed_forms_and_invariants():
+    g = np.random.default_rng(3)
+    n = 257
+    logp, v, h, r = -g.random(n), g.standard_normal(n), g.random(n), g.standard_normal(n)
+    pol, vl, ent = orc.a2c_terms(logp, v, h, r)
+    # definitions through library reductions
+    assert pol == pytest.approx(float(np.mean(logp * (r - v))), rel=1e-13)
+    assert vl == pytest.approx(float(np.mean((r - v) ** 2)), rel=1e-13)
+    assert ent == pytest.approx(float(np.mean(h)), rel=1e-13)
+    # R = V: no policy term, no value loss
+    p0, v0, _ = orc.a2c_terms(logp, v, h, v)
+    assert p0 == 0.0 and v0 == 0.0
+    # uniform policy over A actions: policy term = -ln A * mean advantage
+    A = 18
+    p1, _, _ = orc.a2c_terms(np.full(n, -np.log(A)), v, h, r)
+    assert p1 == pytest.approx(-np.log(A) * float(np.mean(r - v)), rel=1e-12)
+    # order of the transitions does not matter; the advantage enters linearly / quadratically
+    perm = g.permutation(n)
+    assert orc.a2c_terms(logp[perm], v[perm], h[perm], r[perm]) == pytest.approx((pol, vl, ent), rel=1e-12)
+    p2, v2, _ = orc.a2c_terms(logp, 2 * v, h, 2 * r)
+    assert p2 == pytest.approx(2 * pol, rel=1e-12) and v2 == pytest.approx(4 * vl, rel=1e-12)
+    # swapping the sign of the advantage flips the policy term only
+    p3, v3, _ = orc.a2c_terms(logp, r, h, v)
+    assert p3 == pytest.approx(-pol, rel=1e-12) and v3 == pytest.approx(vl, rel=1e-12)
+
+
+def test_evaluate_actions_is_the_distribution_of_the_actor_step():
+    cfg = wl.CONFIGS[1]
+    wt = orc.Weights(wl.make_weights(cfg))
+    n = 6
+    obs = wl.make_obs(cfg, n, batch_index=4)
+    ids = np.arange(n, dtype=np.int32)
+    step = orc.policy_step(wt, obs, ids, 3, 99)
+    ev = orc.evaluate_actions(wt, obs, step["actions"])
+    # the sampled action's log-probability, the value and the entropy are those the actor reported
+    assert np.allclose(ev["logp"], step["logp"], rtol=0, atol=1e-12)
+    assert np.allclose(ev["values"], step["values"], rtol=0, atol=1e-12)
+    assert np.allclose(ev["entropy"], step["entropy"], rtol=0, atol=1e-12)
+    # over all actions the probabilities sum to one and reproduce the entropy
+    for e in range(n):
+        lps = np.array([orc.evaluate_actions(wt, obs[e:e + 1], [a])["logp"][0] for a in range(cfg.A)])
+        assert abs(np.exp(lps).sum() - 1.0) < 1e-12
+        assert abs(-(np.exp(lps) * lps).sum() - ev["entropy"][e]) < 1e-12
+    with pytest.raises(AssertionError):
+        orc.evaluate_actions(wt, obs, np.full(n, cfg.A))
