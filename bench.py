@@ -346,6 +346,28 @@ def run_ours(args) -> None:
         w_ms.append(a.elapsed_time(b))
     wide_ms = float(np.median(w_ms[3:]))
     wide_gbs = (17 * T * Nw + 4 * Nw) / (wide_ms * 1e-3) / 1e9
+    # the learner's sample means (policy term of Eq. 4, value loss, entropy) over the same widened storage
+    # (16 bytes per transition) and over the configuration's own [T, N] storage
+    out3 = torch.empty(3, dtype=torch.float32, device=dev)
+    t_ms = []
+    for i in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_a2c_terms(aw, vw, rw, qw, T * Nw, out3, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        t_ms.append(a.elapsed_time(b))
+    terms_wide_ms = float(np.median(t_ms[3:]))
+    terms_wide_gbs = 16 * T * Nw / (terms_wide_ms * 1e-3) / 1e9
+    t_ms = []
+    for i in range(12):
+        with torch.cuda.stream(s_gae):
+            flush.fill_(i)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_a2c_terms(store[0].logp, store[0].values, store[0].entropy, store[0].ret, T * N, out3, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        t_ms.append(a.elapsed_time(b))
+    terms_us = 1e3 * float(np.median(t_ms[3:]))
     del rw, vw, dw, bw, aw, qw
 
     # ---- dominant kernel and its roofline
@@ -473,6 +495,9 @@ def run_ours(args) -> None:
         "gae": {"us_cold": gae_us, "elems_per_s": T * N / (gae_us * 1e-6), "gbs_cold": gae_bytes / (gae_us * 1e-6) / 1e9,
                 "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
                          "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
+        "learner_terms": {"us_cold": terms_us, "elems": T * N,
+                          "wide": {"elems": T * Nw, "ms": terms_wide_ms, "gbs": terms_wide_gbs,
+                                   "frac_of_hbm": terms_wide_gbs / peaks["hbm_gbs"]}},
         "actor_step_us": 1e3 * ms / (args.steps * T),
         "indexed_actor_step_us": indexed_us,
         "large_batch_actor_step": big,

@@ -131,6 +131,32 @@ hts_status hts_policy_step_indexed(hts_ctx *ctx, const uint8_t *state_buffer, in
                                    int32_t *actions_row, float *logp_row, float *values_row,
                                    float *entropy_row, void *cuda_stream);
 
+/* The learner's re-evaluation of stored transitions (Section 3: the update of Eq. 3/4
+ * needs log pi(a_t|s_t), V(s_t) and H(pi(.|s_t)) under the current parameters for the
+ * actions that were taken).  Same network pass as hts_policy_step, no sampling.
+ *   obs      DEVICE u8  [n,C,H,W]
+ *   actions  DEVICE i32 [n]        the stored actions, each in [0, num_actions)
+ *   logp, values, entropy  DEVICE f32 [n]  out;  logits_or_null DEVICE f32 [n,A] or NULL
+ * For the action hts_policy_step sampled on the same frames and weights the three
+ * outputs equal that step's, bit for bit.  An action outside the range is not used
+ * as an index: that row writes nothing and hts_last_async_error reports INVALID_ARG. */
+hts_status hts_policy_evaluate(hts_ctx *ctx, const uint8_t *obs, const int32_t *actions, int32_t n,
+                               float *logp, float *values, float *entropy, float *logits_or_null,
+                               void *cuda_stream);
+
+/* The three sample means the actor-critic update is built from (Section 3), over
+ * `count` stored transitions in any layout (e.g. the whole [T,N] storage):
+ *   out3[0] = (1/count) sum logp_i (returns_i - values_i)    policy term of Eq. 4 (its
+ *             gradient with the advantage held fixed is Eq. 4's first summand)
+ *   out3[1] = (1/count) sum (returns_i - values_i)^2         value loss J_V
+ *   out3[2] = (1/count) sum entropy_i                        the term Eq. 4 weights by alpha
+ *   logp, values, entropy, returns  DEVICE f32 [count];  out3 DEVICE f32 [3]
+ * Summed in double precision in an order that depends on count alone.  Uses a small
+ * table inside the library: calls on one device must be ordered (one stream, or
+ * events between streams), not concurrent.  Errors: INVALID_ARG, CUDA.            */
+hts_status hts_a2c_terms(const float *logp, const float *values, const float *entropy,
+                         const float *returns, int64_t count, float *out3, void *cuda_stream);
+
 /* Same operation with HOST buffers: copies obs/env_ids/t_per_env to the device,
  * runs the step, copies the four outputs (and logits if asked) back and waits for
  * them.  Uses staging buffers owned by the context (allocated at create time).
@@ -168,7 +194,8 @@ const char *hts_policy_kernel_name(int32_t kernel);
 
 /* Reads and clears the device status word of the context: HTS_ERR_TIMEOUT if a
  * bounded wait ran out, HTS_ERR_INVALID_ARG if hts_policy_step_indexed met a slot
- * outside the pool, HTS_OK if nothing was recorded.  Synchronises with the device. */
+ * outside the pool or hts_policy_evaluate an action outside the range, HTS_OK if
+ * nothing was recorded.  Synchronises with the device.                            */
 hts_status hts_last_async_error(hts_ctx *ctx);
 
 void hts_policy_destroy(hts_ctx *ctx);

@@ -23,6 +23,7 @@ STATUS_NAMES = ["HTS_OK", "HTS_ERR_INVALID_ARG", "HTS_ERR_SHAPE", "HTS_ERR_ALLOC
 WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
                 "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
 EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_indexed", "hts_policy_step_host",
+           "hts_policy_evaluate", "hts_a2c_terms",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
            "hts_gae_host", "hts_policy_step_noalloc", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
@@ -67,6 +68,10 @@ def lib():
         L.hts_policy_step.argtypes = step
         L.hts_policy_step_host.argtypes = step
         L.hts_policy_step_indexed.argtypes = [vp, vp, i32, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp, vp]
+        L.hts_policy_evaluate.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.hts_policy_evaluate.restype = C.c_int
+        L.hts_a2c_terms.argtypes = [vp, vp, vp, vp, C.c_int64, vp, vp]
+        L.hts_a2c_terms.restype = C.c_int
         L.hts_policy_read_activation.argtypes = [vp, i32, i32, vp, vp]
         L.hts_action_uniforms.argtypes = [vp, vp, i32, u64, i32, i32, vp, vp]
         L.hts_policy_profile.argtypes = [vp, i32]
@@ -146,6 +151,16 @@ def hts_policy_step_indexed(ctx, state_buffer, pool, slots, env_ids, t_per_env, 
     _check(lib().hts_policy_step_indexed(ctx, _ptr(state_buffer), int(pool), _ptr(slots), _ptr(env_ids), _ptr(t_per_env),
                                          int(t), int(seed), int(n), _ptr(actions_row), _ptr(logp_row), _ptr(values_row),
                                          _ptr(entropy_row), _stream(stream)), "hts_policy_step_indexed")
+
+
+def hts_policy_evaluate(ctx, obs, actions, n, logp, values, entropy, logits=None, stream=None) -> None:
+    _check(lib().hts_policy_evaluate(ctx, _ptr(obs), _ptr(actions), int(n), _ptr(logp), _ptr(values), _ptr(entropy),
+                                     _ptr(logits), _stream(stream)), "hts_policy_evaluate")
+
+
+def hts_a2c_terms(logp, values, entropy, returns, count, out3, stream=None) -> None:
+    _check(lib().hts_a2c_terms(_ptr(logp), _ptr(values), _ptr(entropy), _ptr(returns), int(count), _ptr(out3),
+                               _stream(stream)), "hts_a2c_terms")
 
 
 def hts_policy_step_host(ctx, obs, env_ids, t_per_env, t, seed, n, actions, logp, values, entropy,

@@ -53,6 +53,7 @@ struct Indexing {
     int pool = 0;
 };
 constexpr int kStatusBadSlot = 100;
+constexpr int kStatusBadAction = 101;     // a stored action outside [0, A) met by the re-evaluation of given actions
 
 // Geometry of the fixed four-layer network for one observation shape.
 struct Geometry {
@@ -93,7 +94,7 @@ hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s);
 hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n, Profiler& prof, cudaStream_t s);
 hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
                     const Indexing& ix, int32_t* actions, float* logp, float* values, float* entropy, float* logits,
-                    cudaStream_t s);
+                    cudaStream_t s, const int32_t* given_actions = nullptr);
 hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s);
 
 // ---- heads + distribution + sampling epilogue (both paths) --------------------------------
@@ -103,7 +104,10 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
                         const float* fc_bias, const float* whead, const float* bhead, int A,
                         const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
                         uint64_t seed, int n, const Indexing& ix, int* status, int32_t* actions, float* logp,
-                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s);
+                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s,
+                        const int32_t* given_actions = nullptr);
+// given_actions != nullptr: no sampling; row e reports log pi(given_actions[e] | s_e) (env_ids, t and seed are
+// not read, actions may be nullptr).  An action outside [0, A) sets kStatusBadAction and the row writes nothing.
 
 hts_status launch_uniforms(const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed, int n,
                            int A, float* out, cudaStream_t s);

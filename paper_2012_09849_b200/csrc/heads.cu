@@ -64,6 +64,7 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
              const float* __restrict__ bhead, int A, const int32_t* __restrict__ env_ids,
              const int32_t* __restrict__ t_per_env, int32_t t_scalar, uint32_t key0, uint32_t key1,
              int n, const int32_t* __restrict__ slots, int pool, int* __restrict__ status,
+             const int32_t* __restrict__ given,
              int32_t* __restrict__ actions, float* __restrict__ logp,
              float* __restrict__ values, float* __restrict__ entropy, float* __restrict__ logits_out,
              float* __restrict__ h_out)
@@ -86,8 +87,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
     __syncthreads();
     const float4* sw4 = s_w4;
     for (int e = blockIdx.x * 8 + wib; e < n; e += gridDim.x * 8) {
-    const uint32_t env = (uint32_t)env_ids[e];                         // issued early: needed only by the sampler
-    const uint32_t tt = (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
+    const uint32_t env = given ? 0u : (uint32_t)env_ids[e];            // issued early: needed only by the sampler
+    const uint32_t tt = given ? 0u : (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
     // hidden vector: lane l owns units 128*i + 4*l + {0..3}, i = 0..3 (float4 everywhere); split
     // partials are summed in index order
     float4 h[4];
@@ -151,6 +152,8 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
     ent = warp_sum(ent);
 
     float best = -INFINITY; int best_a = 0x7fffffff;
+    if (given) best_a = given[e];                       // learner's re-evaluation: the stored action, no sampling
+    else {
     for (int a = lane; a < A; a += 32) {
         const float u = action_uniform(env, tt, a, key0, key1);
         const float score = lg[a] - logf(-logf(u));
@@ -162,15 +165,17 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
         const int oa = __shfl_xor_sync(0xffffffffu, best_a, k);
         if (ob > best || (ob == best && oa < best_a)) { best = ob; best_a = oa; }
     }
+    }
     if (logits_out) for (int a = lane; a < A; a += 32) logits_out[(size_t)e * A + a] = lg[a];
     if (lane == 0) {
         int o = e;                                       // dense, or the row's slot of the storage row
         if (slots) {
             o = slots[e];
-            if ((unsigned)o >= (unsigned)pool) { atomicCAS(status, 0, kStatusBadSlot); o = -1; }
+            if ((unsigned)o >= (unsigned)pool) { if (status) atomicCAS(status, 0, kStatusBadSlot); o = -1; }
         }
+        if ((unsigned)best_a >= (unsigned)A) { if (status) atomicCAS(status, 0, kStatusBadAction); o = -1; }
         if (o >= 0) {
-            actions[o] = best_a;
+            if (actions) actions[o] = best_a;
             logp[o] = lg[best_a] - lse;
             values[o] = lg[A];
             entropy[o] = ent;
@@ -186,7 +191,8 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
                         const float* fc_bias, const float* whead, const float* bhead, int A,
                         const int32_t* env_ids, const int32_t* t_per_env, int32_t t,
                         uint64_t seed, int n, const Indexing& ix, int* status, int32_t* actions, float* logp,
-                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s)
+                        float* values, float* entropy, float* logits, float* h_out, cudaStream_t s,
+                        const int32_t* given_actions)
 {
     if (num_splits < 1 || num_splits > kMaxSplits) return HTS_ERR_INVALID_ARG;
     const size_t smem = (size_t)(A + 1) * kHidden * sizeof(float);
@@ -210,7 +216,7 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
     if (blocks > 2 * sm_count) blocks = 2 * sm_count;
     HTS_CUDA(launch_pdl(heads_kernel, dim3(blocks), dim3(256), smem, s, h_partials, num_splits, split_stride, fc_bias, whead,
                         bhead, A, env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), n, ix.slots,
-                        ix.pool, status, actions, logp, values, entropy, logits, h_out));
+                        ix.pool, status, given_actions, actions, logp, values, entropy, logits, h_out));
     note_launch();
     return HTS_OK;
 }

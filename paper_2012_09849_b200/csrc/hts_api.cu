@@ -90,7 +90,7 @@ hts_status check_step_args(hts_ctx* ctx, const void* obs, const void* env_ids, i
 
 hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const Indexing& ix, const int32_t* env_ids, const int32_t* t_per_env,
                     int32_t t, uint64_t seed, int32_t n, int32_t* actions, float* logp, float* values,
-                    float* entropy, float* logits, cudaStream_t s)
+                    float* entropy, float* logits, cudaStream_t s, const int32_t* given_actions = nullptr)
 {
     const Geometry& g = ctx->g;
     hts_status st;
@@ -98,13 +98,13 @@ hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const Indexing& ix, const 
         st = tc_forward(ctx->tc, obs, ix, n, ctx->prof, s);
         if (st != HTS_OK) return st;
         ctx->prof.begin(K_HEADS, s);
-        st = tc_heads(ctx->tc, env_ids, t_per_env, t, seed, n, ix, actions, logp, values, entropy, logits, s);
+        st = tc_heads(ctx->tc, env_ids, t_per_env, t, seed, n, ix, actions, logp, values, entropy, logits, s, given_actions);
     } else {
         st = ref_forward(g, ctx->rw, ctx->rws, obs, ix, ctx->status, n, ctx->prof, s);
         if (st != HTS_OK) return st;
         ctx->prof.begin(K_HEADS, s);
         st = launch_heads(ctx->rws.h, 1, 0, nullptr, ctx->rw.whead, ctx->rw.bhead, g.A, env_ids, t_per_env, t,
-                          seed, n, ix, ctx->status, actions, logp, values, entropy, logits, nullptr, s);
+                          seed, n, ix, ctx->status, actions, logp, values, entropy, logits, nullptr, s, given_actions);
     }
     if (st != HTS_OK) return st;
     ctx->prof.end(K_HEADS, s);
@@ -216,6 +216,20 @@ hts_status hts_policy_step_indexed(hts_ctx* ctx, const uint8_t* state_buffer, in
                     nullptr, static_cast<cudaStream_t>(cuda_stream));
 }
 
+hts_status hts_policy_evaluate(hts_ctx* ctx, const uint8_t* obs, const int32_t* actions, int32_t n, float* logp,
+                               float* values, float* entropy, float* logits_or_null, void* cuda_stream)
+{
+    if (!ctx || !obs || !actions || !logp || !values || !entropy) return HTS_ERR_INVALID_ARG;
+    if (n < 1 || n > ctx->desc.max_batch) return HTS_ERR_INVALID_ARG;
+    if (!ctx->loaded) return HTS_ERR_UNSUPPORTED;
+    const size_t nn = (size_t)n;
+    const Range in[] = {{obs, nn * ctx->g.C * ctx->g.H * ctx->g.W}, {actions, nn * 4}};
+    const Range outr[] = {{logp, nn * 4}, {values, nn * 4}, {entropy, nn * 4}, {logits_or_null, nn * ctx->g.A * 4}};
+    if (any_overlap(in, 2, outr, 4)) return HTS_ERR_INVALID_ARG;
+    return run_step(ctx, obs, Indexing{}, nullptr, nullptr, 0, 0, n, nullptr, logp, values, entropy, logits_or_null,
+                    static_cast<cudaStream_t>(cuda_stream), actions);
+}
+
 hts_status hts_policy_step_host(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids,
                                 const int32_t* t_per_env, int32_t t, uint64_t seed, int32_t n,
                                 int32_t* actions, float* logp, float* values, float* entropy,
@@ -269,7 +283,7 @@ hts_status hts_last_async_error(hts_ctx* ctx)
     HTS_CUDA(cudaMemcpy(&word, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (word != 0) {
         HTS_CUDA(cudaMemset(ctx->status, 0, sizeof(int)));
-        return word == kStatusBadSlot ? HTS_ERR_INVALID_ARG : HTS_ERR_TIMEOUT;
+        return (word == kStatusBadSlot || word == kStatusBadAction) ? HTS_ERR_INVALID_ARG : HTS_ERR_TIMEOUT;
     }
     return HTS_OK;
 }

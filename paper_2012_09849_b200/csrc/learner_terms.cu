@@ -1,0 +1,109 @@
+// The three sample means of the actor-critic update (Section 3): the policy term of Eq. 4,
+// (1/|D|) sum log pi(a|s) (R - V), the value loss J_V = (1/|D|) sum (R - V)^2 and the mean entropy.
+//
+// HBM-bound (16 bytes per transition).  Each block sums a contiguous range in double precision in a
+// fixed order (thread-strided float4 loads, shuffle tree, warp order), writes its partial and takes a
+// ticket; the block that draws the last ticket adds the partials in block order.  The grid is a
+// function of the count alone, so the result does not depend on timing or on the device's load.
+#include "common.cuh"
+
+namespace hts {
+namespace {
+
+constexpr int kBlocksMax = 1024;
+constexpr int kThreads = 256;
+constexpr int kPerThread = 8;             // elements a thread covers before another block is worth its launch
+
+// Partials and the ticket counter live in the library image: calls on one device must not overlap.
+__device__ double g_partial[kBlocksMax][3];
+__device__ unsigned int g_ticket;
+
+__device__ __forceinline__ double warp_sum_d(double v)
+{
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+    return v;
+}
+
+__global__ void __launch_bounds__(kThreads)
+a2c_terms_kernel(const float* __restrict__ logp, const float* __restrict__ values, const float* __restrict__ entropy,
+                 const float* __restrict__ returns, long long count, long long per_block, float* __restrict__ out)
+{
+    __shared__ double s_part[kThreads / 32][3];
+    __shared__ bool s_last;
+    const long long lo = (long long)blockIdx.x * per_block;               // per_block is a multiple of 4
+    long long hi = lo + per_block; hi = hi > count ? count : hi;
+    double pol = 0.0, vl = 0.0, ent = 0.0;
+    const bool vec = (((uintptr_t)logp | (uintptr_t)values | (uintptr_t)entropy | (uintptr_t)returns) & 15u) == 0;
+    if (vec) {
+        const long long q_lo = lo >> 2, q_hi = hi >> 2;                    // whole float4 groups of the range
+        const float4* l4 = reinterpret_cast<const float4*>(logp);
+        const float4* v4 = reinterpret_cast<const float4*>(values);
+        const float4* h4 = reinterpret_cast<const float4*>(entropy);
+        const float4* r4 = reinterpret_cast<const float4*>(returns);
+        auto add = [&](const float4& l, const float4& v, const float4& h, const float4& r) {
+            const double a0 = (double)r.x - v.x, a1 = (double)r.y - v.y, a2 = (double)r.z - v.z, a3 = (double)r.w - v.w;
+            pol += (double)l.x * a0; pol += (double)l.y * a1; pol += (double)l.z * a2; pol += (double)l.w * a3;
+            vl += a0 * a0; vl += a1 * a1; vl += a2 * a2; vl += a3 * a3;
+            ent += (double)h.x; ent += (double)h.y; ent += (double)h.z; ent += (double)h.w;
+        };
+        long long q = q_lo + threadIdx.x;
+        for (; q + kThreads < q_hi; q += 2 * kThreads) {                   // eight loads in flight per thread
+            const float4 la = l4[q], va = v4[q], ha = h4[q], ra = r4[q];
+            const float4 lb = l4[q + kThreads], vb = v4[q + kThreads], hb = h4[q + kThreads], rb = r4[q + kThreads];
+            add(la, va, ha, ra);
+            add(lb, vb, hb, rb);
+        }
+        if (q < q_hi) add(l4[q], v4[q], h4[q], r4[q]);
+        for (long long i = (q_hi << 2) + threadIdx.x; i < hi; i += kThreads) {   // the last block's ragged tail
+            const double a = (double)returns[i] - values[i];
+            pol += (double)logp[i] * a; vl += a * a; ent += (double)entropy[i];
+        }
+    } else {
+        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
+            const double a = (double)returns[i] - values[i];
+            pol += (double)logp[i] * a; vl += a * a; ent += (double)entropy[i];
+        }
+    }
+    pol = warp_sum_d(pol); vl = warp_sum_d(vl); ent = warp_sum_d(ent);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_part[warp][0] = pol; s_part[warp][1] = vl; s_part[warp][2] = ent; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0, c = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) { a += s_part[w][0]; b += s_part[w][1]; c += s_part[w][2]; }
+        g_partial[blockIdx.x][0] = a; g_partial[blockIdx.x][1] = b; g_partial[blockIdx.x][2] = c;
+        __threadfence();
+        s_last = atomicAdd(&g_ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {
+        __threadfence();
+        double a = 0.0, b = 0.0, c = 0.0;
+        for (unsigned k = 0; k < gridDim.x; ++k) {                           // block order, whatever the arrival order
+            a += *(volatile double*)&g_partial[k][0]; b += *(volatile double*)&g_partial[k][1]; c += *(volatile double*)&g_partial[k][2];
+        }
+        const double inv = 1.0 / (double)count;
+        out[0] = (float)(a * inv); out[1] = (float)(b * inv); out[2] = (float)(c * inv);
+        g_ticket = 0;                                                        // ready for the next call
+    }
+}
+
+}  // namespace
+}  // namespace hts
+
+extern "C" hts_status hts_a2c_terms(const float* logp, const float* values, const float* entropy, const float* returns,
+                                    int64_t count, float* out3, void* cuda_stream)
+{
+    using namespace hts;
+    if (!logp || !values || !entropy || !returns || !out3 || count < 1) return HTS_ERR_INVALID_ARG;
+    long long blocks = (count + (long long)kThreads * kPerThread - 1) / ((long long)kThreads * kPerThread);
+    if (blocks > kBlocksMax) blocks = kBlocksMax;
+    long long per_block = (count + blocks - 1) / blocks;
+    per_block = (per_block + 3) / 4 * 4;
+    blocks = (count + per_block - 1) / per_block;
+    a2c_terms_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        logp, values, entropy, returns, (long long)count, per_block, out3);
+    HTS_LAUNCH_CHECK("a2c_terms_kernel");
+    return HTS_OK;
+}

@@ -424,10 +424,10 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
 
 hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env, int32_t tt, uint64_t seed, int n,
                     const Indexing& ix, int32_t* actions, float* logp, float* values, float* entropy, float* logits,
-                    cudaStream_t s)
+                    cudaStream_t s, const int32_t* given_actions)
 {
     return launch_heads(t->hpart, t->splits, (size_t)t->max_batch * 512, t->bfc, t->whead, t->bhead, t->g.A, env_ids,
-                        t_per_env, tt, seed, n, ix, t->status, actions, logp, values, entropy, logits, t->h, s);
+                        t_per_env, tt, seed, n, ix, t->status, actions, logp, values, entropy, logits, t->h, s, given_actions);
 }
 
 hts_status tc_read_activation(TcState* t, int layer, int n, float* out, cudaStream_t s)
