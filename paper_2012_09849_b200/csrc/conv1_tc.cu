@@ -359,13 +359,15 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_a = tmem_slot, tmem_d = tmem_slot + 128;
+    if (threadIdx.x == 0) {                                   // the filter does not depend on the previous kernel
+        mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
+        for (int g = 0; g < 4; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
+    }
     pdl_wait();
     pdl_trigger();
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
-            for (int g = 0; g < 4; ++g) tma_load_2d(sm + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
             const size_t chan = (size_t)pl.H * pl.W, frame = chan * pl.C;
             PixelWalk first;
             first.init(128u * blockIdx.x, step, pl.H1, pl.W1);

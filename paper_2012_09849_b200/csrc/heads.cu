@@ -100,7 +100,7 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
         for (int sp = 0; sp < kMaxSplits; ++sp)
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                part[sp][i] = (sp < num_splits) ? hp[sp * stride4 + 32 * i] : make_float4(0.f, 0.f, 0.f, 0.f);
+                part[sp][i] = hp[(sp < num_splits ? sp : 0) * stride4 + 32 * i];   // unconditional: all loads in flight at once
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             float4 v = part[0][i];
@@ -115,10 +115,12 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
             if (h_out) reinterpret_cast<float4*>(h_out + (size_t)e * kHidden)[32 * i + lane] = v;
         }
     }
-    for (int o0 = 0; o0 <= A; o0 += 4) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    // Eight outputs per pass: their dot products and shuffle trees are independent, so the pass costs
+    // little more than one tree's latency.  Each output keeps its own fixed summation order.
+    for (int o0 = 0; o0 <= A; o0 += 8) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 8; ++j) {
             const int o = (o0 + j <= A) ? o0 + j : A;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -130,9 +132,11 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
 #pragma unroll
         for (int m = 16; m > 0; m >>= 1)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], m);
-        if (lane < 4 && o0 + lane <= A) {
-            const float mine = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
+            for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], m);
+        if (lane < 8 && o0 + lane <= A) {
+            float mine = acc[0];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) mine = lane == j ? acc[j] : mine;
             s_out[wib][o0 + lane] = mine + s_bhead[o0 + lane];
         }
     }
