@@ -44,6 +44,26 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 
 inline int conv_out(int extent, int k, int s) { return (extent - k) / s + 1; }
 
+// Kernel attributes (dynamic shared memory, carve-out) belong to a device, and so does the SM count:
+// the launchers keep their "already set" marks per device, indexed by this slot.
+constexpr int kDeviceSlots = 64;
+inline int device_slot()
+{
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess) { cudaGetLastError(); d = 0; }
+    return (d >= 0 && d < kDeviceSlots) ? d : 0;
+}
+inline int device_sm_count(int slot)
+{
+    static int count[kDeviceSlots] = {};
+    if (!count[slot]) {
+        int d = 0, c = 0;
+        if (cudaGetDevice(&d) == cudaSuccess && cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, d) == cudaSuccess) count[slot] = c;
+        else cudaGetLastError();
+    }
+    return count[slot] > 0 ? count[slot] : 1;
+}
+
 // Executor-facing addressing of a step (state buffer -> actors -> storage row, Section 4.1): row e of the
 // batch reads frame slots[e] of a pool of `pool` frames and writes its outputs at index slots[e].
 // slots == nullptr: frames and outputs are dense, row e at index e.  A slot outside [0, pool) is

@@ -573,12 +573,11 @@ hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __ha
 hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, const Indexing& ix, int n,
                         const float* bias, const float* inv_scale, __half* out, int* status, cudaStream_t s)
 {
-    static int sm_count = 0, max_smem_set = 0;
-    if (!sm_count) {
-        int dev = 0;
-        HTS_CUDA(cudaGetDevice(&dev));
-        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    }
+    const int dev = device_slot();
+    const int sm_count = device_sm_count(dev);
+    static int smem_set_by_device[kDeviceSlots] = {}, ts_smem_set_by_device[kDeviceSlots] = {};
+    int& max_smem_set = smem_set_by_device[dev];
+    int& ts_smem_set = ts_smem_set_by_device[dev];
     if (max_smem_set < pl.smem_bytes) {
         HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
         HTS_CUDA(cudaFuncSetAttribute(conv1_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes));
@@ -591,7 +590,6 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, cons
         max_smem_set = pl.smem_bytes;
     }
     if (pl.ts && (long)n * pl.H1 * pl.W1 < (1L << 31) - 128 * 2 * sm_count) {
-        static int ts_smem_set = 0;
         if (ts_smem_set < pl.ts_smem_bytes) {
             HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<84>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.ts_smem_bytes));
             HTS_CUDA(cudaFuncSetAttribute(conv1_ts_kernel<84>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));

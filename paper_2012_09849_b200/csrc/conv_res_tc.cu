@@ -175,12 +175,10 @@ template <int TAPS, int CPT>
 hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight_map, const ConvResParams& p,
                            cudaStream_t s)
 {
-    static int sm_count = 0, smem_set = 0;
-    if (!sm_count) {
-        int dev = 0;
-        HTS_CUDA(cudaGetDevice(&dev));
-        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    }
+    const int dev = device_slot();
+    const int sm_count = device_sm_count(dev);
+    static int smem_set_by_device[kDeviceSlots] = {};
+    int& smem_set = smem_set_by_device[dev];
     constexpr int NST = CPT == 2 ? 4 : 6;        // activation tiles in the ring: two being multiplied, the rest in flight
     const int smem = 1024 + TAPS * CPT * kChunkBytes + NST * CPT * p.tile_rows * 128;
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;

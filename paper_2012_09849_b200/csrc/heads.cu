@@ -200,8 +200,12 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
 {
     if (num_splits < 1 || num_splits > kMaxSplits) return HTS_ERR_INVALID_ARG;
     const size_t smem = (size_t)(A + 1) * kHidden * sizeof(float);
-    static size_t smem_set = 48 * 1024;
-    static bool carveout_set = false;
+    const int dev = device_slot();
+    static size_t smem_set_by_device[kDeviceSlots] = {};
+    static bool carveout_set_by_device[kDeviceSlots] = {};
+    size_t& smem_set = smem_set_by_device[dev];
+    bool& carveout_set = carveout_set_by_device[dev];
+    if (smem_set == 0) smem_set = 48 * 1024;            // what a kernel may use without asking
     if (!carveout_set) {
         HTS_CUDA(cudaFuncSetAttribute(heads_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         carveout_set = true;
@@ -210,12 +214,7 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
         HTS_CUDA(cudaFuncSetAttribute(heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         smem_set = smem;
     }
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        HTS_CUDA(cudaGetDevice(&dev));
-        HTS_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-    }
+    const int sm_count = device_sm_count(dev);
     int blocks = (n + 7) / 8;
     if (blocks > 2 * sm_count) blocks = 2 * sm_count;
     HTS_CUDA(launch_pdl(heads_kernel, dim3(blocks), dim3(256), smem, s, h_partials, num_splits, split_stride, fc_bias, whead,

@@ -371,8 +371,11 @@ hts_status hts_gae_host(const float* rewards, const float* values, const uint8_t
 {
     hts_status st = check_gae_args(rewards, values, dones, bootstrap, gamma, lambda, T, N, advantages, returns);
     if (st != HTS_OK) return st;
-    static char* stage = nullptr;
-    static size_t stage_bytes = 0;
+    static char* stage_by_device[kDeviceSlots] = {};
+    static size_t stage_bytes_by_device[kDeviceSlots] = {};
+    const int dev = device_slot();
+    char*& stage = stage_by_device[dev];
+    size_t& stage_bytes = stage_bytes_by_device[dev];
     const size_t tn = (size_t)T * N;
     const size_t tn4 = (tn * 4 + 255) / 256 * 256, tn1 = (tn + 255) / 256 * 256, n4 = ((size_t)N * 4 + 255) / 256 * 256;
     const size_t need = 4 * tn4 + tn1 + n4;

@@ -280,7 +280,8 @@ template <int BN, int EPI>
 hts_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& p, dim3 grid, cudaStream_t s)
 {
     constexpr int smem = STAGES * (A_BYTES + BN * BK * 2) + 1024;
-    static bool attr_set = false;
+    static bool attr_set_by_device[kDeviceSlots] = {};
+    bool& attr_set = attr_set_by_device[device_slot()];
     if (!attr_set) {
         HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HTS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
