@@ -112,10 +112,10 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         if (lane == 0) {
             mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
             for (int g = 0; g < 4 * CPT; ++g) tma_load_2d(s_w + g * kChunkBytes, &tmW, g * 64, 0, &w_bar);
-            int it = 0;
-            for (int u = blockIdx.x; u < units; u += gridDim.x, ++it) {
-                const int s = it % NU;
-                if (!mbar_wait(&u8_empty[s], (((uint32_t)(it / NU)) & 1u) ^ 1u, abortp, p.status, 11)) break;
+            int s = 0;                                    // staged band and the parity of its current use: a ring
+            uint32_t sph = 0;                             // walked with counters (NU is not a compile-time constant)
+            for (int u = blockIdx.x; u < units; u += gridDim.x) {
+                if (!mbar_wait(&u8_empty[s], sph ^ 1u, abortp, p.status, 11)) break;
                 const int env = u / pl.bands, band = u - env * pl.bands;
                 const int r0 = 4 * band * pl.R;
                 int rows = pl.H - r0; rows = rows > band_in_rows ? band_in_rows : rows;
@@ -125,6 +125,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 uint8_t* dst = s_u8 + s * pl.u8_stage_bytes;
                 for (int c = 0; c < pl.C; ++c)
                     bulk_load(dst + c * band_in_rows * pl.W, src + (size_t)c * pl.H * pl.W, bytes, &u8_full[s]);
+                if (++s == NU) { s = 0; sph ^= 1u; }
             }
         }
     } else if (warp == 1 || warp == 14) {
@@ -172,12 +173,13 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         int it = 0, pb = 0;
         uint32_t pph = 0;
         bool alive = true;
+        int s = 0;
+        uint32_t sph = 0;
         for (int u = blockIdx.x; alive && u < units; u += gridDim.x, ++it) {
-            const int s = it % NU;
             const int band = u % pl.bands;
             int in_rows = pl.H - 4 * band * pl.R; in_rows = in_rows > band_in_rows ? band_in_rows : in_rows;
             const int pixels = (in_rows >> 2) * pl.Ws;   // space-to-depth pixels present in this band
-            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 14)) break;
+            if (!mbar_wait_warp(&u8_full[s], sph, abortp, p.status, 14)) break;
             const uint8_t* src = s_u8 + s * pl.u8_stage_bytes + src_q;
 #pragma unroll
             for (int pln = 0; pln < CPT; ++pln) {
@@ -203,6 +205,7 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 if (++pb == NP) { pb = 0; pph ^= 1u; }
             }
             if (alive) mbar_arrive(&u8_empty[s]);
+            if (++s == NU) { s = 0; sph ^= 1u; }
         }
     } else if (warp < 14) {
         // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1 and add the two accumulators
@@ -371,10 +374,10 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
             const size_t chan = (size_t)pl.H * pl.W, frame = chan * pl.C;
             PixelWalk first;
             first.init(128u * blockIdx.x, step, pl.H1, pl.W1);
-            int it = 0;
-            for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, first.advance(pl.H1, pl.W1)) {
-                const int s = it % NU;
-                if (!mbar_wait(&u8_empty[s], (((uint32_t)(it / NU)) & 1u) ^ 1u, abortp, p.status, 31)) break;
+            int s = 0;                                    // staged tile and the parity of its current use
+            uint32_t sph = 0;
+            for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, first.advance(pl.H1, pl.W1)) {
+                if (!mbar_wait(&u8_empty[s], sph ^ 1u, abortp, p.status, 31)) break;
                 int nA, nB;
                 ts_rows(pl, p.n, first.e, first.y, first.x, nA, nB);
                 const uint32_t bytesA = (uint32_t)((4 * nA + 4) * W), bytesB = nB ? (uint32_t)((4 * nB + 4) * W) : 0u;
@@ -387,6 +390,7 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                     const uint8_t* srcB = p.obs + frame_of(p, first.e + 1) * frame;
                     for (int c = 0; c < pl.C; ++c) bulk_load(dst + c * chan_bytes + bytesA, srcB + c * chan, bytesB, &u8_full[s]);
                 }
+                if (++s == NU) { s = 0; sph ^= 1u; }
             }
         }
     } else if (warp == 1 || warp == 14) {
@@ -422,16 +426,16 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         PixelWalk first, mine;
         first.init(128u * blockIdx.x, step, pl.H1, pl.W1);
         mine.init(128u * blockIdx.x + (uint32_t)m, step, pl.H1, pl.W1);
-        int it = 0;
+        int it = 0, s = 0;
+        uint32_t sph = 0;
         for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++it, first.advance(pl.H1, pl.W1), mine.advance(pl.H1, pl.W1)) {
-            const int s = it % NU;
             // Staged input row under this pixel's window: four rows per output row since the tile's
             // first one, plus the four extra rows that close the first environment's part.  Rows past
             // the end of the batch read the start of the buffer: their results are never stored.
             const int segB = mine.e != first.e;
             const int row = 4 * ((segB ? pl.H1 : 0) + mine.y - first.y + segB + h);
             const int off = mine.e < p.n ? row * W + 4 * mine.x : 0;
-            if (!mbar_wait_warp(&u8_full[s], ((uint32_t)(it / NU)) & 1u, abortp, p.status, 35)) break;
+            if (!mbar_wait_warp(&u8_full[s], sph, abortp, p.status, 35)) break;
             const uint8_t* src = s_u8 + s * pl.ts_stage_bytes + off;
             bool alive = true;
 #pragma unroll
@@ -452,6 +456,7 @@ conv1_ts_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 mbar_arrive(&q_full[2 * h + dx]);
             }
             if (!alive) break;
+            if (++s == NU) { s = 0; sph ^= 1u; }
         }
     } else if (warp < 14) {
         // ---- epilogue: warps 10..13 read TMEM lane quarters 2,3,0,1
