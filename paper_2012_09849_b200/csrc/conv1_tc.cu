@@ -168,8 +168,17 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
         const int qq = tid & 7, slot = tid >> 3;         // slot 0..31
         const int src_q = ((qq >> 1) * band_in_rows + 2 * (qq & 1)) * pl.W;     // channel (qq>>1) of a plane, row pair (qq&1)
         const int plane_src = 4 * band_in_rows * pl.W;                          // four channels per plane
-        const int ys0 = slot / pl.Ws, xs0 = slot - ys0 * pl.Ws;                  // first pixel of this thread
-        const int dys = 32 / pl.Ws, dxs = 32 - dys * pl.Ws;                      // step of 32 pixels on the grid
+        // This thread's pixels slot, slot + 32, ... of a plane never change: their source and
+        // destination offsets are worked out once (the converter warps are bound by instruction issue).
+        constexpr int kIters = 7;                        // tile_rows <= 200 pixels / 32 per pass
+        int soff[kIters], doff[kIters];
+#pragma unroll
+        for (int i = 0; i < kIters; ++i) {
+            const int ps = slot + 32 * i;
+            const int ys = ps / pl.Ws, xs = ps - ys * pl.Ws;
+            soff[i] = (4 * ys) * pl.W + 4 * xs;
+            doff[i] = ps * 128 + ((qq ^ (ps & 7)) << 4);  // chunk qq of row ps, 128-byte swizzle: qq ^ (ps % 8)
+        }
         int it = 0, pb = 0;
         uint32_t pph = 0;
         bool alive = true;
@@ -186,19 +195,17 @@ conv1_tc_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
                 if (!mbar_wait_warp(&plane_empty[pb], pph ^ 1u, abortp, p.status, 17)) { alive = false; break; }
                 uint8_t* dplane = s_tile + pb * plane_bytes;
                 const uint8_t* splane = src + pln * plane_src;
-                int ys = ys0, xs = xs0;
-#pragma unroll 5
-                for (int ps = slot; ps < pixels; ps += 32) {
-                    const uint8_t* s0 = splane + (4 * ys) * pl.W + 4 * xs;
-                    const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
-                    const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
-                    uint4 o;
-                    u8x4_to_h4(w0, o.x, o.y);
-                    u8x4_to_h4(w1, o.z, o.w);
-                    // chunk qq of row ps, 128-byte swizzle: qq ^ (ps % 8)
-                    *reinterpret_cast<uint4*>(dplane + ps * 128 + ((qq ^ (ps & 7)) << 4)) = o;
-                    xs += dxs; ys += dys;
-                    if (xs >= pl.Ws) { xs -= pl.Ws; ++ys; }
+#pragma unroll
+                for (int i = 0; i < kIters; ++i) {
+                    if (slot + 32 * i < pixels) {
+                        const uint8_t* s0 = splane + soff[i];
+                        const uint32_t w0 = *reinterpret_cast<const uint32_t*>(s0);
+                        const uint32_t w1 = *reinterpret_cast<const uint32_t*>(s0 + pl.W);
+                        uint4 o;
+                        u8x4_to_h4(w0, o.x, o.y);
+                        u8x4_to_h4(w1, o.z, o.w);
+                        *reinterpret_cast<uint4*>(dplane + doff[i]) = o;
+                    }
                 }
                 fence_async_proxy();                     // plane stores -> visible to the tensor core's reads
                 mbar_arrive(&plane_full[pb]);
