@@ -222,3 +222,23 @@ def a2c_terms(logp, values, entropy, returns):
         vl += adv * adv
         ent += entropy[i]
     return pol / count, vl / count, ent / count
+
+
+def delayed_update(theta, grad, sq_avg, lr: float, alpha: float, eps: float, precondition: bool = True):
+    """One learner update of Section 4.1 "Delayed gradient", Eq. 5: theta_{j+1} = theta_j + eta * d, where the
+    gradient of J-hat was taken at theta_{j-1} by the caller.  With RMSProp (Appendix F tables: momentum 0, epsilon
+    given) d = g / (sqrt(v) + eps) and v <- alpha v + (1 - alpha) g^2 (Tieleman & Hinton's rule, denominator as in
+    the table's epsilon); without it d = g.  fp64.  -> (theta_next, sq_avg_next)."""
+    theta, grad, sq_avg = (np.asarray(a, dtype=np.float64) for a in (theta, grad, sq_avg))
+    assert theta.shape == grad.shape == sq_avg.shape
+    out_t, out_v = np.empty_like(theta), np.empty_like(sq_avg)
+    ft, fg, fv, ot, ov = theta.ravel(), grad.ravel(), sq_avg.ravel(), out_t.ravel(), out_v.ravel()
+    for i in range(ft.size):
+        if precondition:
+            v = alpha * fv[i] + (1.0 - alpha) * fg[i] * fg[i]
+            d = fg[i] / (np.sqrt(v) + eps)
+        else:
+            v, d = fv[i], fg[i]
+        ov[i] = v
+        ot[i] = ft[i] + lr * d
+    return out_t, out_v

@@ -70,3 +70,56 @@ def test_evaluate_actions_is_the_distribution_of_the_actor_step():
         assert abs(-(np.exp(lps) * lps).sum() - ev["entropy"][e]) < 1e-12
     with pytest.raises(AssertionError):
         orc.evaluate_actions(wt, obs, np.full(n, cfg.A))
+
+
+def _gold_update():
+    path = os.path.join(os.path.dirname(GOLD), "delayed_update_worked_example.txt")
+    rows, exp = [], {}
+    for line in open(path, encoding="utf-8"):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        if line.startswith("expected"):
+            k, *v = line.split()
+            exp[k] = np.array([float(x) for x in v])
+        else:
+            rows.append([float(x) for x in line.split()])
+    return np.array(rows), exp
+
+
+def test_delayed_update_worked_example():
+    a, exp = _gold_update()
+    t, v = orc.delayed_update(a[:, 0], a[:, 1], a[:, 2], lr=0.5, alpha=0.75, eps=0.5)
+    assert np.array_equal(v, exp["expected_v"])
+    assert np.allclose(t, exp["expected_theta"], rtol=0, atol=1e-16)
+    t2, v2 = orc.delayed_update(a[:, 0], a[:, 1], a[:, 2], lr=0.5, alpha=0.75, eps=0.5, precondition=False)
+    assert np.array_equal(t2, exp["expected_plain"]) and np.array_equal(v2, a[:, 2])
+
+
+def test_delayed_update_closed_forms():
+    g = np.random.default_rng(11)
+    n = 300
+    theta, grad, v = g.standard_normal(n), g.standard_normal(n), g.random(n)
+    # zero gradient: parameters stay, the running average decays by alpha
+    t0, v0 = orc.delayed_update(theta, np.zeros(n), v, 0.1, 0.9, 1e-5)
+    assert np.array_equal(t0, theta) and np.allclose(v0, 0.9 * v, rtol=1e-15)
+    # alpha = 0: v' = g^2, so the step is eta * g / (|g| + eps), bounded by eta and of the gradient's sign
+    t1, v1 = orc.delayed_update(theta, grad, v, 0.1, 0.0, 1e-5)
+    assert np.allclose(v1, grad ** 2, rtol=1e-15)
+    assert np.allclose(t1 - theta, 0.1 * grad / (np.abs(grad) + 1e-5), rtol=1e-12)
+    assert np.all(np.abs(t1 - theta) < 0.1) and np.all(np.sign(t1 - theta) == np.sign(grad))
+    # library expression of the rule; ascent direction (Eq. 5 adds the gradient of the objective)
+    t2, v2 = orc.delayed_update(theta, grad, v, 0.01, 0.99, 0.01)
+    vv = 0.99 * v + 0.01 * grad ** 2
+    assert np.allclose(v2, vv, rtol=1e-15) and np.allclose(t2, theta + 0.01 * grad / (np.sqrt(vv) + 0.01), rtol=1e-13)
+    # constant gradient: v converges to g^2 and the step to eta * g / (|g| + eps)
+    tt, vv = theta.copy(), np.zeros(n)
+    for _ in range(2000):
+        prev = tt
+        tt, vv = orc.delayed_update(tt, grad, vv, 0.001, 0.99, 1e-3)
+    assert np.allclose(vv, grad ** 2, rtol=1e-6)
+    assert np.allclose(tt - prev, 0.001 * grad / (np.abs(grad) + 1e-3), rtol=1e-6)
+    # plain Eq. 5 is linear in the gradient
+    ta, _ = orc.delayed_update(theta, grad, v, 0.3, 0.9, 1e-5, precondition=False)
+    tb, _ = orc.delayed_update(theta, 2 * grad, v, 0.3, 0.9, 1e-5, precondition=False)
+    assert np.allclose(tb - theta, 2 * (ta - theta), rtol=1e-13)
