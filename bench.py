@@ -368,7 +368,19 @@ def run_ours(args) -> None:
         b.record(s_gae); torch.cuda.synchronize()
         t_ms.append(a.elapsed_time(b))
     terms_us = 1e3 * float(np.median(t_ms[3:]))
-    del rw, vw, dw, bw, aw, qw
+    # the learner's parameter update (Eq. 5 with RMSProp scaling) over a parameter vector of the widened size
+    upd_ms = []
+    hb = torch.empty(T * Nw, dtype=torch.bfloat16, device=dev)
+    aw.zero_(); qw.fill_(1e-4)
+    for i in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_delayed_update(aw, vw, qw, T * Nw, 7e-4, 0.99, 1e-5, hb, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        upd_ms.append(a.elapsed_time(b))
+    upd_wide_ms = float(np.median(upd_ms[3:]))
+    upd_gbs = 22 * T * Nw / (upd_wide_ms * 1e-3) / 1e9
+    del rw, vw, dw, bw, aw, qw, hb
 
     # ---- dominant kernel and its roofline
     macs = layer_macs(cfg)
@@ -498,6 +510,7 @@ def run_ours(args) -> None:
         "learner_terms": {"us_cold": terms_us, "elems": T * N,
                           "wide": {"elems": T * Nw, "ms": terms_wide_ms, "gbs": terms_wide_gbs,
                                    "frac_of_hbm": terms_wide_gbs / peaks["hbm_gbs"]}},
+        "delayed_update": {"elems": T * Nw, "ms": upd_wide_ms, "gbs": upd_gbs, "frac_of_hbm": upd_gbs / peaks["hbm_gbs"]},
         "actor_step_us": 1e3 * ms / (args.steps * T),
         "indexed_actor_step_us": indexed_us,
         "large_batch_actor_step": big,

@@ -157,6 +157,21 @@ hts_status hts_policy_evaluate(hts_ctx *ctx, const uint8_t *obs, const int32_t *
 hts_status hts_a2c_terms(const float *logp, const float *values, const float *entropy,
                          const float *returns, int64_t count, float *out3, void *cuda_stream);
 
+/* One learner update with the one-step-delayed gradient (Section 4.1, Eq. 5):
+ *   theta <- theta + lr * d,  where grad is the gradient of the objective J-hat that
+ * the caller took at the PREVIOUS parameters (the ones the rollout was collected
+ * with).  With sq_avg given, d is RMSProp-scaled as in the hyper-parameter tables of
+ * Appendix F (momentum 0):  v <- alpha v + (1-alpha) grad^2,  d = grad / (sqrt(v) + eps);
+ * with sq_avg NULL, d = grad (Eq. 5 as printed; alpha and eps unused).
+ *   theta, grad, sq_avg  DEVICE f32 [count] (theta and sq_avg updated in place)
+ *   theta_bf16_or_null   DEVICE bf16 [count] or NULL  out: the new parameters rounded to
+ *                        bf16 in the same pass, ready for hts_policy_load_weights
+ * The sign is ascent on J-hat; pass the negated gradient of a loss.  0 <= alpha <= 1,
+ * eps > 0, lr finite.  Errors: INVALID_ARG, CUDA.                                  */
+hts_status hts_delayed_update(float *theta, const float *grad, float *sq_avg_or_null, int64_t count,
+                              float lr, float alpha, float eps, void *theta_bf16_or_null,
+                              void *cuda_stream);
+
 /* Same operation with HOST buffers: copies obs/env_ids/t_per_env to the device,
  * runs the step, copies the four outputs (and logits if asked) back and waits for
  * them.  Uses staging buffers owned by the context (allocated at create time).

@@ -5,6 +5,7 @@
 // fixed order (thread-strided float4 loads, shuffle tree, warp order), writes its partial and takes a
 // ticket; the block that draws the last ticket adds the partials in block order.  The grid is a
 // function of the count alone, so the result does not depend on timing or on the device's load.
+#include <cmath>
 #include "common.cuh"
 
 namespace hts {
@@ -105,5 +106,86 @@ extern "C" hts_status hts_a2c_terms(const float* logp, const float* values, cons
     a2c_terms_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         logp, values, entropy, returns, (long long)count, per_block, out3);
     HTS_LAUNCH_CHECK("a2c_terms_kernel");
+    return HTS_OK;
+}
+
+// ---- the learner's parameter update (Section 4.1 "Delayed gradient", Eq. 5) ---------------------------------
+// theta_{j+1} = theta_j + eta * d with the gradient taken (by the caller) at theta_{j-1}.  With the RMSProp
+// scaling of the hyper-parameter tables (momentum 0): v <- alpha v + (1 - alpha) g^2, d = g / (sqrt(v) + eps);
+// without it d = g.  Elementwise and HBM-bound: 20 bytes per parameter, 22 with the bf16 copy that the actor's
+// hts_policy_load_weights takes, written in the same pass.
+namespace hts {
+namespace {
+
+template <bool PRECOND>
+__device__ __forceinline__ float update_one(float theta, float g, float& v, float lr, float alpha, float eps)
+{
+    float d = g;
+    if (PRECOND) {
+        v = fmaf(alpha, v, (1.0f - alpha) * g * g);
+        d = g / (sqrtf(v) + eps);
+    }
+    return fmaf(lr, d, theta);
+}
+
+// Four parameters per thread and pass when every array is 16-byte aligned (8 for the bf16 copy).
+template <bool PRECOND, bool VEC>
+__global__ void __launch_bounds__(256)
+delayed_update_kernel(float* __restrict__ theta, const float* __restrict__ grad, float* __restrict__ sq_avg,
+                      long long count, float lr, float alpha, float eps, __nv_bfloat16* __restrict__ theta_bf16)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    long long done = 0;
+    if (VEC) {
+        const long long quads = count >> 2;
+        for (long long q = tid; q < quads; q += stride) {
+            const float4 g = reinterpret_cast<const float4*>(grad)[q];
+            float4 t = reinterpret_cast<float4*>(theta)[q];
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (PRECOND) v = reinterpret_cast<float4*>(sq_avg)[q];
+            t.x = update_one<PRECOND>(t.x, g.x, v.x, lr, alpha, eps); t.y = update_one<PRECOND>(t.y, g.y, v.y, lr, alpha, eps);
+            t.z = update_one<PRECOND>(t.z, g.z, v.z, lr, alpha, eps); t.w = update_one<PRECOND>(t.w, g.w, v.w, lr, alpha, eps);
+            reinterpret_cast<float4*>(theta)[q] = t;
+            if (PRECOND) reinterpret_cast<float4*>(sq_avg)[q] = v;
+            if (theta_bf16) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+                reinterpret_cast<uint2*>(theta_bf16)[q] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+            }
+        }
+        done = quads << 2;
+    }
+    for (long long i = done + tid; i < count; i += stride) {
+        float v = PRECOND ? sq_avg[i] : 0.f;
+        const float t = update_one<PRECOND>(theta[i], grad[i], v, lr, alpha, eps);
+        theta[i] = t;
+        if (PRECOND) sq_avg[i] = v;
+        if (theta_bf16) theta_bf16[i] = __float2bfloat16_rn(t);
+    }
+}
+
+}  // namespace
+}  // namespace hts
+
+extern "C" hts_status hts_delayed_update(float* theta, const float* grad, float* sq_avg_or_null, int64_t count,
+                                         float lr, float alpha, float eps, void* theta_bf16_or_null, void* cuda_stream)
+{
+    using namespace hts;
+    if (!theta || !grad || count < 1) return HTS_ERR_INVALID_ARG;
+    if (!(lr == lr) || std::isinf(lr)) return HTS_ERR_INVALID_ARG;
+    if (sq_avg_or_null && (!(alpha >= 0.f && alpha <= 1.f) || !(eps > 0.f) || std::isinf(eps))) return HTS_ERR_INVALID_ARG;
+    long long blocks = (count + 256 * 4 - 1) / (256 * 4);
+    const long long cap = 16LL * device_sm_count(device_slot());
+    if (blocks > cap) blocks = cap;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    __nv_bfloat16* tb = static_cast<__nv_bfloat16*>(theta_bf16_or_null);
+    const bool vec = (((uintptr_t)theta | (uintptr_t)grad | (uintptr_t)sq_avg_or_null) & 15u) == 0 && ((uintptr_t)tb & 7u) == 0;
+    const unsigned gb = (unsigned)blocks;
+    const long long n = (long long)count;
+    if (sq_avg_or_null && vec) delayed_update_kernel<true, true><<<gb, 256, 0, s>>>(theta, grad, sq_avg_or_null, n, lr, alpha, eps, tb);
+    else if (sq_avg_or_null) delayed_update_kernel<true, false><<<gb, 256, 0, s>>>(theta, grad, sq_avg_or_null, n, lr, alpha, eps, tb);
+    else if (vec) delayed_update_kernel<false, true><<<gb, 256, 0, s>>>(theta, grad, nullptr, n, lr, alpha, eps, tb);
+    else delayed_update_kernel<false, false><<<gb, 256, 0, s>>>(theta, grad, nullptr, n, lr, alpha, eps, tb);
+    HTS_LAUNCH_CHECK("delayed_update_kernel");
     return HTS_OK;
 }

@@ -129,3 +129,67 @@ def test_a2c_terms_unaligned_views_and_refusals():
     L = hts.lib()
     assert L.hts_a2c_terms(8, 16, 24, 32, 0, 40, None) == 1
     assert L.hts_a2c_terms(None, 16, 24, 32, 4, 40, None) == 1
+
+
+@pytest.mark.parametrize("count", [1, 5, 1025, 1693875, (1 << 22) + 3])
+def test_delayed_update_against_oracle(count):
+    g = np.random.default_rng(count)
+    theta = g.standard_normal(count, dtype=np.float32)
+    grad = (g.standard_normal(count, dtype=np.float32) * 0.1).astype(np.float32)
+    v = (g.random(count, dtype=np.float32) * 0.01).astype(np.float32)
+    lr, alpha, eps = np.float32(7e-4), np.float32(0.99), np.float32(1e-5)
+    d_t, d_g, d_v = (torch.from_numpy(a.copy()).cuda() for a in (theta, grad, v))
+    d_b = torch.empty(count, dtype=torch.bfloat16, device="cuda")
+    hts.hts_delayed_update(d_t, d_g, d_v, count, lr, alpha, eps, d_b)
+    torch.cuda.synchronize()
+    n_ref = min(count, 20000)                                   # the oracle is a Python loop
+    rt, rv = orc.delayed_update(theta[:n_ref], grad[:n_ref], v[:n_ref], float(lr), float(alpha), float(eps))
+    got_t, got_v = d_t.cpu().numpy(), d_v.cpu().numpy()
+    assert np.all(np.abs(got_v[:n_ref] - rv) <= 1e-6 * np.maximum(np.abs(rv), 1e-8))
+    assert np.all(np.abs(got_t[:n_ref] - rt) <= 1e-6 * np.maximum(np.abs(rt), 1e-3))
+    # at size: the rule through fp64 library expressions
+    vv = float(alpha) * v.astype(np.float64) + (1.0 - float(alpha)) * grad.astype(np.float64) ** 2
+    tt = theta + float(lr) * grad / (np.sqrt(vv) + float(eps))
+    assert np.all(np.abs(got_t - tt) <= 1e-6 * np.maximum(np.abs(tt), 1e-3))
+    # the bf16 copy is the new fp32 parameter rounded to nearest even
+    assert torch.equal(d_b, d_t.to(torch.bfloat16))
+    # plain Eq. 5
+    d_t2 = torch.from_numpy(theta.copy()).cuda()
+    hts.hts_delayed_update(d_t2, d_g, None, count, 0.5, 0.0, 0.0)
+    torch.cuda.synchronize()
+    scale = np.maximum(np.maximum(np.abs(theta), np.abs(0.5 * grad)), 1e-3)         # fp32 rounding of the larger operand
+    assert np.all(np.abs(d_t2.cpu().numpy() - (theta + 0.5 * grad.astype(np.float64))) <= 1e-6 * scale)
+
+
+def test_delayed_update_golden_and_refusals():
+    path = os.path.join(os.path.dirname(GOLD), "delayed_update_worked_example.txt")
+    rows, exp = [], {}
+    for line in open(path, encoding="utf-8"):
+        line = line.split("#")[0].strip()
+        if line.startswith("expected"):
+            k, *vals = line.split()
+            exp[k] = np.array([float(x) for x in vals])
+        elif line:
+            rows.append([float(x) for x in line.split()])
+    a = np.array(rows, dtype=np.float32)
+    d_t, d_g, d_v = (torch.from_numpy(a[:, i].copy()).cuda() for i in range(3))
+    hts.hts_delayed_update(d_t, d_g, d_v, 4, 0.5, 0.75, 0.5)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_v.cpu().numpy(), exp["expected_v"].astype(np.float32))
+    assert np.allclose(d_t.cpu().numpy(), exp["expected_theta"], rtol=2e-7, atol=0)
+    # views that are only 4-byte aligned take the scalar path and give the same numbers
+    g = np.random.default_rng(2)
+    n = 1003
+    base = [torch.from_numpy(g.standard_normal(n + 1, dtype=np.float32)).abs().cuda() for _ in range(3)]
+    al = [b[:n].clone() for b in base]
+    un = [b.clone()[1:] for b in [torch.cat([b[:1], b[:n]]) for b in base]]
+    hts.hts_delayed_update(al[0], al[1], al[2], n, 0.01, 0.9, 1e-3)
+    hts.hts_delayed_update(un[0], un[1], un[2], n, 0.01, 0.9, 1e-3)
+    torch.cuda.synchronize()
+    assert torch.equal(al[0], un[0]) and torch.equal(al[2], un[2])
+    L = hts.lib()
+    assert L.hts_delayed_update(None, 8, 16, 4, 0.1, 0.9, 1e-5, None, None) == 1
+    assert L.hts_delayed_update(8, 16, 24, 0, 0.1, 0.9, 1e-5, None, None) == 1
+    assert L.hts_delayed_update(8, 16, 24, 4, 0.1, 1.5, 1e-5, None, None) == 1
+    assert L.hts_delayed_update(8, 16, 24, 4, 0.1, 0.9, 0.0, None, None) == 1
+    assert L.hts_delayed_update(8, 16, 24, 4, float("nan"), 0.9, 1e-5, None, None) == 1
