@@ -11,7 +11,7 @@
 namespace hts {
 namespace {
 
-constexpr int kBlocksMax = 1024;
+constexpr int kBlocksMax = 2048;
 constexpr int kThreads = 256;
 constexpr int kPerThread = 8;             // elements a thread covers before another block is worth its launch
 
@@ -49,13 +49,14 @@ a2c_terms_kernel(const float* __restrict__ logp, const float* __restrict__ value
             ent += (double)h.x; ent += (double)h.y; ent += (double)h.z; ent += (double)h.w;
         };
         long long q = q_lo + threadIdx.x;
-        for (; q + kThreads < q_hi; q += 2 * kThreads) {                   // eight loads in flight per thread
-            const float4 la = l4[q], va = v4[q], ha = h4[q], ra = r4[q];
-            const float4 lb = l4[q + kThreads], vb = v4[q + kThreads], hb = h4[q + kThreads], rb = r4[q + kThreads];
-            add(la, va, ha, ra);
-            add(lb, vb, hb, rb);
+        for (; q + 3 * kThreads < q_hi; q += 4 * kThreads) {               // sixteen loads in flight per thread
+            float4 l[4], v[4], h[4], r[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { l[u] = l4[q + u * kThreads]; v[u] = v4[q + u * kThreads]; h[u] = h4[q + u * kThreads]; r[u] = r4[q + u * kThreads]; }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) add(l[u], v[u], h[u], r[u]);
         }
-        if (q < q_hi) add(l4[q], v4[q], h4[q], r4[q]);
+        for (; q < q_hi; q += kThreads) add(l4[q], v4[q], h4[q], r4[q]);
         for (long long i = (q_hi << 2) + threadIdx.x; i < hi; i += kThreads) {   // the last block's ragged tail
             const double a = (double)returns[i] - values[i];
             pol += (double)logp[i] * a; vl += a * a; ent += (double)entropy[i];
@@ -78,15 +79,20 @@ a2c_terms_kernel(const float* __restrict__ logp, const float* __restrict__ value
         s_last = atomicAdd(&g_ticket, 1u) == gridDim.x - 1;
     }
     __syncthreads();
-    if (s_last && threadIdx.x == 0) {
+    if (s_last && threadIdx.x < 32) {
+        // lane l adds partials l, l + 32, ... in that order, then the lanes are folded by a shuffle tree: an order
+        // fixed by the grid size, whatever the arrival order of the blocks
         __threadfence();
         double a = 0.0, b = 0.0, c = 0.0;
-        for (unsigned k = 0; k < gridDim.x; ++k) {                           // block order, whatever the arrival order
+        for (unsigned k = threadIdx.x; k < gridDim.x; k += 32) {
             a += *(volatile double*)&g_partial[k][0]; b += *(volatile double*)&g_partial[k][1]; c += *(volatile double*)&g_partial[k][2];
         }
-        const double inv = 1.0 / (double)count;
-        out[0] = (float)(a * inv); out[1] = (float)(b * inv); out[2] = (float)(c * inv);
-        g_ticket = 0;                                                        // ready for the next call
+        a = warp_sum_d(a); b = warp_sum_d(b); c = warp_sum_d(c);
+        if (threadIdx.x == 0) {
+            const double inv = 1.0 / (double)count;
+            out[0] = (float)(a * inv); out[1] = (float)(b * inv); out[2] = (float)(c * inv);
+            g_ticket = 0;                                                    // ready for the next call
+        }
     }
 }
 
