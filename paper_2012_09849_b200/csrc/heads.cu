@@ -86,7 +86,9 @@ heads_kernel(const float* __restrict__ h_partials, int num_splits, size_t split_
     pdl_trigger();
     __syncthreads();
     const float4* sw4 = s_w4;
-    for (int e = blockIdx.x * 8 + wib; e < n; e += gridDim.x * 8) {
+    // rows are dealt block-first (row g goes to block g % gridDim.x), so a batch of fewer rows than warps on
+    // the device still spreads over every block
+    for (int e = wib * gridDim.x + blockIdx.x; e < n; e += gridDim.x * 8) {
     const uint32_t env = given ? 0u : (uint32_t)env_ids[e];            // issued early: needed only by the sampler
     const uint32_t tt = given ? 0u : (uint32_t)(t_per_env ? t_per_env[e] : t_scalar);
     // hidden vector: lane l owns units 128*i + 4*l + {0..3}, i = 0..3 (float4 everywhere); split
@@ -215,8 +217,8 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
         smem_set = smem;
     }
     const int sm_count = device_sm_count(dev);
-    int blocks = (n + 7) / 8;
-    if (blocks > 2 * sm_count) blocks = 2 * sm_count;
+    int blocks = n <= 8 * sm_count ? sm_count : 2 * sm_count;     // one block per SM until every warp has a row
+    if (blocks > n) blocks = n;
     HTS_CUDA(launch_pdl(heads_kernel, dim3(blocks), dim3(256), smem, s, h_partials, num_splits, split_stride, fc_bias, whead,
                         bhead, A, env_ids, t_per_env, t, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), n, ix.slots,
                         ix.pool, status, given_actions, actions, logp, values, entropy, logits, h_out));
