@@ -33,7 +33,7 @@ import hts_workloads as wl  # noqa: E402
 WORKLOAD = 3                       # hts_workloads.CONFIGS index
 # dram__bytes_read.sum + dram__bytes_write.sum of one conv1_ts_kernel<84> launch at this workload (n = 1024),
 # from the ncu capture summarised in profiles/actor_step_cfg3_n1024.md; reported only for that kernel
-CONV1_DRAM_TRAFFIC_BYTES = 28959744 + 60160
+CONV1_DRAM_TRAFFIC_BYTES = 28958720 + 126976
 METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
 UNIT = "env-steps/s"
 SEED = 0x5EED
