@@ -242,3 +242,35 @@ def delayed_update(theta, grad, sq_avg, lr: float, alpha: float, eps: float, pre
         ov[i] = v
         ot[i] = ft[i] + lr * d
     return out_t, out_v
+
+
+def ppo_terms(logp_new, logp_old, values, entropy, advantages, returns, clip: float, normalize: bool):
+    """Sample means of the clipped surrogate of proximal policy optimisation (Schulman et al. 2017, Eq. 7), the
+    algorithm HTS-RL is run with on the football scenarios (Section 5, "Ours (PPO)"):
+        rho_i = exp(logp_new_i - logp_old_i),   A_i the advantage (optionally standardised over the batch:
+        (A - mean) / (std + 1e-8), population std),
+        surrogate = mean(min(rho A, clip(rho, 1 - clip, 1 + clip) A)),
+    plus the value loss mean((R - V)^2), the mean entropy and the fraction of samples with |rho - 1| > clip.
+    fp64.  -> (surrogate, value_loss, mean_entropy, clip_fraction)."""
+    lp, lo, v, h, a, r = (np.asarray(x, dtype=np.float64).ravel() for x in (logp_new, logp_old, values, entropy, advantages, returns))
+    n = lp.size
+    assert n > 0 and all(x.size == n for x in (lo, v, h, a, r)) and clip > 0
+    if normalize:
+        mean = 0.0
+        for i in range(n):
+            mean += a[i]
+        mean /= n
+        var = 0.0
+        for i in range(n):
+            var += (a[i] - mean) ** 2
+        std = np.sqrt(var / n)
+        a = (a - mean) / (std + 1e-8)
+    sur = vl = ent = frac = 0.0
+    for i in range(n):
+        rho = np.exp(lp[i] - lo[i])
+        clipped = min(max(rho, 1.0 - clip), 1.0 + clip)
+        sur += min(rho * a[i], clipped * a[i])
+        vl += (r[i] - v[i]) ** 2
+        ent += h[i]
+        frac += 1.0 if abs(rho - 1.0) > clip else 0.0
+    return sur / n, vl / n, ent / n, frac / n

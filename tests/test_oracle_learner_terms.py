@@ -123,3 +123,52 @@ def test_delayed_update_closed_forms():
     ta, _ = orc.delayed_update(theta, grad, v, 0.3, 0.9, 1e-5, precondition=False)
     tb, _ = orc.delayed_update(theta, 2 * grad, v, 0.3, 0.9, 1e-5, precondition=False)
     assert np.allclose(tb - theta, 2 * (ta - theta), rtol=1e-13)
+
+
+def _gold_ppo():
+    path = os.path.join(os.path.dirname(GOLD), "ppo_terms_worked_example.txt")
+    rows, exp = [], None
+    for line in open(path, encoding="utf-8"):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        if line.startswith("expected"):
+            exp = [float(x) for x in line.split()[1:]]
+        else:
+            rows.append([float(x) for x in line.split()])
+    return np.array(rows), exp
+
+
+def test_ppo_terms_worked_example():
+    a, exp = _gold_ppo()
+    lp_old = np.full(len(a), -1.5)
+    got = orc.ppo_terms(lp_old + np.log(a[:, 0]), lp_old, a[:, 2], a[:, 4], a[:, 1], a[:, 3], 0.25, False)
+    assert np.allclose(got, exp, rtol=1e-15, atol=0)
+
+
+def test_ppo_terms_closed_forms():
+    g = np.random.default_rng(8)
+    n = 400
+    lo = -g.random(n) * 2
+    v, r, h, adv = g.standard_normal(n), g.standard_normal(n), g.random(n), g.standard_normal(n)
+    # identical policies: rho = 1, the surrogate is the mean advantage and nothing is clipped
+    s, vl, ent, frac = orc.ppo_terms(lo, lo, v, h, adv, r, 0.2, False)
+    assert s == pytest.approx(float(np.mean(adv)), rel=1e-13) and frac == 0.0
+    assert vl == pytest.approx(float(np.mean((r - v) ** 2)), rel=1e-13) and ent == pytest.approx(float(np.mean(h)), rel=1e-13)
+    # standardised advantages have mean 0: with rho = 1 the surrogate vanishes; the standardisation is shift/scale free
+    s0, *_ = orc.ppo_terms(lo, lo, v, h, adv, r, 0.2, True)
+    assert abs(s0) < 1e-12
+    ln = lo + 0.3 * g.standard_normal(n)
+    a1 = orc.ppo_terms(ln, lo, v, h, adv, r, 0.2, True)
+    a2 = orc.ppo_terms(ln, lo, v, h, 5.0 * adv + 3.0, r, 0.2, True)
+    assert np.allclose(a1, a2, rtol=1e-7)
+    # the surrogate never exceeds the unclipped importance-weighted mean, and equals it for a huge clip range
+    rho = np.exp(ln - lo)
+    s1, _, _, f1 = orc.ppo_terms(ln, lo, v, h, adv, r, 0.2, False)
+    assert s1 <= float(np.mean(rho * adv)) + 1e-15 and 0.0 < f1 < 1.0
+    assert f1 == pytest.approx(float(np.mean(np.abs(rho - 1.0) > 0.2)), rel=1e-15)
+    s2, _, _, f2 = orc.ppo_terms(ln, lo, v, h, adv, r, 1e6, False)
+    assert s2 == pytest.approx(float(np.mean(rho * adv)), rel=1e-13) and f2 == 0.0
+    # library expression
+    ref = float(np.mean(np.minimum(rho * adv, np.clip(rho, 0.8, 1.2) * adv)))
+    assert s1 == pytest.approx(ref, rel=1e-13)
