@@ -368,6 +368,19 @@ def run_ours(args) -> None:
         b.record(s_gae); torch.cuda.synchronize()
         t_ms.append(a.elapsed_time(b))
     terms_us = 1e3 * float(np.median(t_ms[3:]))
+    # the PPO form (clipped surrogate, standardised advantages: two passes over the advantages + one over all six arrays)
+    out4 = torch.empty(4, dtype=torch.float32, device=dev)
+    x1, x2 = torch.zeros_like(vw), torch.zeros_like(vw)          # six distinct arrays
+    t_ms = []
+    for i in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_ppo_terms(aw, x1, vw, qw, rw, x2, T * Nw, 0.2, True, out4, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        t_ms.append(a.elapsed_time(b))
+    ppo_wide_ms = float(np.median(t_ms[3:]))
+    ppo_wide_gbs = 32 * T * Nw / (ppo_wide_ms * 1e-3) / 1e9
+    del x1, x2
     # the learner's parameter update (Eq. 5 with RMSProp scaling) over a parameter vector of the widened size
     upd_ms = []
     hb = torch.empty(T * Nw, dtype=torch.bfloat16, device=dev)
@@ -509,7 +522,10 @@ def run_ours(args) -> None:
                          "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
         "learner_terms": {"us_cold": terms_us, "elems": T * N,
                           "wide": {"elems": T * Nw, "ms": terms_wide_ms, "gbs": terms_wide_gbs,
-                                   "frac_of_hbm": terms_wide_gbs / peaks["hbm_gbs"]}},
+                                   "frac_of_hbm": terms_wide_gbs / peaks["hbm_gbs"]},
+                          "ppo_wide": {"elems": T * Nw, "ms": ppo_wide_ms, "gbs": ppo_wide_gbs,
+                                       "frac_of_hbm": ppo_wide_gbs / peaks["hbm_gbs"],
+                                       "bytes_per_elem": "24 (six arrays) + 2 x 4 (advantage mean and variance passes)"}},
         "delayed_update": {"elems": T * Nw, "ms": upd_wide_ms, "gbs": upd_gbs, "frac_of_hbm": upd_gbs / peaks["hbm_gbs"]},
         "actor_step_us": 1e3 * ms / (args.steps * T),
         "indexed_actor_step_us": indexed_us,

@@ -157,6 +157,22 @@ hts_status hts_policy_evaluate(hts_ctx *ctx, const uint8_t *obs, const int32_t *
 hts_status hts_a2c_terms(const float *logp, const float *values, const float *entropy,
                          const float *returns, int64_t count, float *out3, void *cuda_stream);
 
+/* The same for proximal policy optimisation, the algorithm HTS-RL is run with on the
+ * football scenarios (Section 5, "Ours (PPO)"; objective of Schulman et al. 2017, Eq. 7):
+ *   rho_i   = exp(logp_new_i - logp_old_i)
+ *   A_i     = advantages_i, or (advantages_i - mean) / (std + 1e-8) over the batch
+ *             (population std) if normalize_advantages != 0
+ *   out4[0] = (1/count) sum min(rho_i A_i, clip(rho_i, 1-clip, 1+clip) A_i)   clipped surrogate
+ *   out4[1] = (1/count) sum (returns_i - values_i)^2                          value loss
+ *   out4[2] = (1/count) sum entropy_i
+ *   out4[3] = fraction of samples with |rho_i - 1| > clip
+ *   all inputs DEVICE f32 [count]; out4 DEVICE f32 [4]; clip > 0.
+ * Summation, ordering and the non-concurrency rule as for hts_a2c_terms.            */
+hts_status hts_ppo_terms(const float *logp_new, const float *logp_old, const float *values,
+                         const float *entropy, const float *advantages, const float *returns,
+                         int64_t count, float clip, int32_t normalize_advantages, float *out4,
+                         void *cuda_stream);
+
 /* One learner update with the one-step-delayed gradient (Section 4.1, Eq. 5):
  *   theta <- theta + lr * d,  where grad is the gradient of the objective J-hat that
  * the caller took at the PREVIOUS parameters (the ones the rollout was collected

@@ -23,7 +23,7 @@ STATUS_NAMES = ["HTS_OK", "HTS_ERR_INVALID_ARG", "HTS_ERR_SHAPE", "HTS_ERR_ALLOC
 WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
                 "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
 EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_indexed", "hts_policy_step_host",
-           "hts_policy_evaluate", "hts_a2c_terms", "hts_delayed_update",
+           "hts_policy_evaluate", "hts_a2c_terms", "hts_ppo_terms", "hts_delayed_update",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
            "hts_gae_host", "hts_policy_step_noalloc", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
@@ -72,6 +72,8 @@ def lib():
         L.hts_policy_evaluate.restype = C.c_int
         L.hts_a2c_terms.argtypes = [vp, vp, vp, vp, C.c_int64, vp, vp]
         L.hts_a2c_terms.restype = C.c_int
+        L.hts_ppo_terms.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int64, f32, i32, vp, vp]
+        L.hts_ppo_terms.restype = C.c_int
         L.hts_delayed_update.argtypes = [vp, vp, vp, C.c_int64, f32, f32, f32, vp, vp]
         L.hts_delayed_update.restype = C.c_int
         L.hts_policy_read_activation.argtypes = [vp, i32, i32, vp, vp]
@@ -163,6 +165,11 @@ def hts_policy_evaluate(ctx, obs, actions, n, logp, values, entropy, logits=None
 def hts_a2c_terms(logp, values, entropy, returns, count, out3, stream=None) -> None:
     _check(lib().hts_a2c_terms(_ptr(logp), _ptr(values), _ptr(entropy), _ptr(returns), int(count), _ptr(out3),
                                _stream(stream)), "hts_a2c_terms")
+
+
+def hts_ppo_terms(logp_new, logp_old, values, entropy, advantages, returns, count, clip, normalize, out4, stream=None) -> None:
+    _check(lib().hts_ppo_terms(_ptr(logp_new), _ptr(logp_old), _ptr(values), _ptr(entropy), _ptr(advantages), _ptr(returns),
+                               int(count), float(clip), int(bool(normalize)), _ptr(out4), _stream(stream)), "hts_ppo_terms")
 
 
 def hts_delayed_update(theta, grad, sq_avg, count, lr, alpha, eps, theta_bf16=None, stream=None) -> None:

@@ -1,9 +1,12 @@
-// The three sample means of the actor-critic update (Section 3): the policy term of Eq. 4,
-// (1/|D|) sum log pi(a|s) (R - V), the value loss J_V = (1/|D|) sum (R - V)^2 and the mean entropy.
+// Sample means over the stored transitions that the learner's objectives are built from:
+//   hts_a2c_terms  Section 3: the policy term of Eq. 4, (1/|D|) sum log pi(a|s) (R - V), the value loss
+//                  J_V = (1/|D|) sum (R - V)^2 and the mean entropy;
+//   hts_ppo_terms  the clipped surrogate of proximal policy optimisation (Schulman et al. 2017, Eq. 7), the
+//                  algorithm the football runs of Section 5 use, with the same value loss and entropy.
 //
-// HBM-bound (16 bytes per transition).  Each block sums a contiguous range in double precision in a
+// HBM-bound (16 to 24 bytes per transition).  Each block sums a contiguous range in double precision in a
 // fixed order (thread-strided float4 loads, shuffle tree, warp order), writes its partial and takes a
-// ticket; the block that draws the last ticket adds the partials in block order.  The grid is a
+// ticket; the block that draws the last ticket adds the partials in a fixed order.  The grid is a
 // function of the count alone, so the result does not depend on timing or on the device's load.
 #include <cmath>
 #include "common.cuh"
@@ -14,10 +17,13 @@ namespace {
 constexpr int kBlocksMax = 2048;
 constexpr int kThreads = 256;
 constexpr int kPerThread = 8;             // elements a thread covers before another block is worth its launch
+constexpr int kMaxSums = 4;
 
-// Partials and the ticket counter live in the library image: calls on one device must not overlap.
-__device__ double g_partial[kBlocksMax][3];
+// Partials, the ticket counter and the advantage statistics live in the library image: calls on one device
+// must not overlap.
+__device__ double g_partial[kBlocksMax][kMaxSums];
 __device__ unsigned int g_ticket;
+__device__ double g_adv_stats[2];         // mean and 1 / (std + 1e-8) of the advantages (hts_ppo_terms)
 
 __device__ __forceinline__ double warp_sum_d(double v)
 {
@@ -26,55 +32,49 @@ __device__ __forceinline__ double warp_sum_d(double v)
     return v;
 }
 
+// An Op names NS sums, how four consecutive elements (float4 group q) or one element i add to them, whether
+// its arrays allow float4 loads, and what the last block does with the totals.
+template <class Op>
 __global__ void __launch_bounds__(kThreads)
-a2c_terms_kernel(const float* __restrict__ logp, const float* __restrict__ values, const float* __restrict__ entropy,
-                 const float* __restrict__ returns, long long count, long long per_block, float* __restrict__ out)
+sums_kernel(const Op op, long long count, long long per_block)
 {
-    __shared__ double s_part[kThreads / 32][3];
+    constexpr int NS = Op::NS;
+    __shared__ double s_part[kThreads / 32][NS];
     __shared__ bool s_last;
     const long long lo = (long long)blockIdx.x * per_block;               // per_block is a multiple of 4
     long long hi = lo + per_block; hi = hi > count ? count : hi;
-    double pol = 0.0, vl = 0.0, ent = 0.0;
-    const bool vec = (((uintptr_t)logp | (uintptr_t)values | (uintptr_t)entropy | (uintptr_t)returns) & 15u) == 0;
-    if (vec) {
+    double acc[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) acc[k] = 0.0;
+    if (op.aligned16()) {
         const long long q_lo = lo >> 2, q_hi = hi >> 2;                    // whole float4 groups of the range
-        const float4* l4 = reinterpret_cast<const float4*>(logp);
-        const float4* v4 = reinterpret_cast<const float4*>(values);
-        const float4* h4 = reinterpret_cast<const float4*>(entropy);
-        const float4* r4 = reinterpret_cast<const float4*>(returns);
-        auto add = [&](const float4& l, const float4& v, const float4& h, const float4& r) {
-            const double a0 = (double)r.x - v.x, a1 = (double)r.y - v.y, a2 = (double)r.z - v.z, a3 = (double)r.w - v.w;
-            pol += (double)l.x * a0; pol += (double)l.y * a1; pol += (double)l.z * a2; pol += (double)l.w * a3;
-            vl += a0 * a0; vl += a1 * a1; vl += a2 * a2; vl += a3 * a3;
-            ent += (double)h.x; ent += (double)h.y; ent += (double)h.z; ent += (double)h.w;
-        };
         long long q = q_lo + threadIdx.x;
-        for (; q + 3 * kThreads < q_hi; q += 4 * kThreads) {               // sixteen loads in flight per thread
-            float4 l[4], v[4], h[4], r[4];
+        for (; q + 3 * kThreads < q_hi; q += 4 * kThreads) {               // four groups per array in flight per thread
+            typename Op::Quad g[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { l[u] = l4[q + u * kThreads]; v[u] = v4[q + u * kThreads]; h[u] = h4[q + u * kThreads]; r[u] = r4[q + u * kThreads]; }
+            for (int u = 0; u < 4; ++u) g[u] = op.load4(q + u * kThreads);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) add(l[u], v[u], h[u], r[u]);
+            for (int u = 0; u < 4; ++u) op.add4(g[u], acc);
         }
-        for (; q < q_hi; q += kThreads) add(l4[q], v4[q], h4[q], r4[q]);
-        for (long long i = (q_hi << 2) + threadIdx.x; i < hi; i += kThreads) {   // the last block's ragged tail
-            const double a = (double)returns[i] - values[i];
-            pol += (double)logp[i] * a; vl += a * a; ent += (double)entropy[i];
-        }
+        for (; q < q_hi; q += kThreads) op.add4(op.load4(q), acc);
+        for (long long i = (q_hi << 2) + threadIdx.x; i < hi; i += kThreads) op.add1(i, acc);   // the last block's ragged tail
     } else {
-        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
-            const double a = (double)returns[i] - values[i];
-            pol += (double)logp[i] * a; vl += a * a; ent += (double)entropy[i];
-        }
+        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) op.add1(i, acc);
     }
-    pol = warp_sum_d(pol); vl = warp_sum_d(vl); ent = warp_sum_d(ent);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (lane == 0) { s_part[warp][0] = pol; s_part[warp][1] = vl; s_part[warp][2] = ent; }
+#pragma unroll
+    for (int k = 0; k < NS; ++k) {
+        acc[k] = warp_sum_d(acc[k]);
+        if (lane == 0) s_part[warp][k] = acc[k];
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
-        double a = 0.0, b = 0.0, c = 0.0;
-        for (int w = 0; w < kThreads / 32; ++w) { a += s_part[w][0]; b += s_part[w][1]; c += s_part[w][2]; }
-        g_partial[blockIdx.x][0] = a; g_partial[blockIdx.x][1] = b; g_partial[blockIdx.x][2] = c;
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            double a = 0.0;
+            for (int w = 0; w < kThreads / 32; ++w) a += s_part[w][k];
+            g_partial[blockIdx.x][k] = a;
+        }
         __threadfence();
         s_last = atomicAdd(&g_ticket, 1u) == gridDim.x - 1;
     }
@@ -83,18 +83,142 @@ a2c_terms_kernel(const float* __restrict__ logp, const float* __restrict__ value
         // lane l adds partials l, l + 32, ... in that order, then the lanes are folded by a shuffle tree: an order
         // fixed by the grid size, whatever the arrival order of the blocks
         __threadfence();
-        double a = 0.0, b = 0.0, c = 0.0;
-        for (unsigned k = threadIdx.x; k < gridDim.x; k += 32) {
-            a += *(volatile double*)&g_partial[k][0]; b += *(volatile double*)&g_partial[k][1]; c += *(volatile double*)&g_partial[k][2];
-        }
-        a = warp_sum_d(a); b = warp_sum_d(b); c = warp_sum_d(c);
+        double tot[NS];
+#pragma unroll
+        for (int k = 0; k < NS; ++k) tot[k] = 0.0;
+        for (unsigned b = threadIdx.x; b < gridDim.x; b += 32)
+#pragma unroll
+            for (int k = 0; k < NS; ++k) tot[k] += *(volatile double*)&g_partial[b][k];
+#pragma unroll
+        for (int k = 0; k < NS; ++k) tot[k] = warp_sum_d(tot[k]);
         if (threadIdx.x == 0) {
-            const double inv = 1.0 / (double)count;
-            out[0] = (float)(a * inv); out[1] = (float)(b * inv); out[2] = (float)(c * inv);
-            g_ticket = 0;                                                    // ready for the next call
+            op.finish(tot, count);
+            g_ticket = 0;                                                    // ready for the next launch
         }
     }
 }
+
+template <class Op>
+hts_status launch_sums(const Op& op, long long count, cudaStream_t s, const char* name)
+{
+    long long blocks = (count + (long long)kThreads * kPerThread - 1) / ((long long)kThreads * kPerThread);
+    if (blocks > kBlocksMax) blocks = kBlocksMax;
+    long long per_block = (count + blocks - 1) / blocks;
+    per_block = (per_block + 3) / 4 * 4;
+    blocks = (count + per_block - 1) / per_block;
+    sums_kernel<Op><<<(unsigned)blocks, kThreads, 0, s>>>(op, count, per_block);
+    HTS_LAUNCH_CHECK(name);
+    return HTS_OK;
+}
+
+inline bool all_aligned16(std::initializer_list<const void*> ps)
+{
+    uintptr_t x = 0;
+    for (const void* p : ps) x |= (uintptr_t)p;
+    return (x & 15u) == 0;
+}
+
+struct A2cOp {
+    static constexpr int NS = 3;
+    const float *logp, *values, *entropy, *returns;
+    float* out;
+    bool vec;
+    struct Quad { float4 l, v, h, r; };
+    __device__ bool aligned16() const { return vec; }
+    __device__ Quad load4(long long q) const
+    {
+        return Quad{reinterpret_cast<const float4*>(logp)[q], reinterpret_cast<const float4*>(values)[q],
+                    reinterpret_cast<const float4*>(entropy)[q], reinterpret_cast<const float4*>(returns)[q]};
+    }
+    __device__ static void one(float l, float v, float h, float r, double* acc)
+    {
+        const double a = (double)r - v;
+        acc[0] += (double)l * a; acc[1] += a * a; acc[2] += (double)h;
+    }
+    __device__ void add4(const Quad& g, double* acc) const
+    {
+        one(g.l.x, g.v.x, g.h.x, g.r.x, acc); one(g.l.y, g.v.y, g.h.y, g.r.y, acc);
+        one(g.l.z, g.v.z, g.h.z, g.r.z, acc); one(g.l.w, g.v.w, g.h.w, g.r.w, acc);
+    }
+    __device__ void add1(long long i, double* acc) const { one(logp[i], values[i], entropy[i], returns[i], acc); }
+    __device__ void finish(const double* tot, long long count) const
+    {
+        const double inv = 1.0 / (double)count;
+        out[0] = (float)(tot[0] * inv); out[1] = (float)(tot[1] * inv); out[2] = (float)(tot[2] * inv);
+    }
+};
+
+// first and second pass over the advantages: mean, then 1 / (population std + 1e-8)
+struct AdvMeanOp {
+    static constexpr int NS = 1;
+    const float* adv;
+    bool vec;
+    using Quad = float4;
+    __device__ bool aligned16() const { return vec; }
+    __device__ Quad load4(long long q) const { return reinterpret_cast<const float4*>(adv)[q]; }
+    __device__ void add4(const Quad& g, double* acc) const { acc[0] += (double)g.x; acc[0] += (double)g.y; acc[0] += (double)g.z; acc[0] += (double)g.w; }
+    __device__ void add1(long long i, double* acc) const { acc[0] += (double)adv[i]; }
+    __device__ void finish(const double* tot, long long count) const { g_adv_stats[0] = tot[0] / (double)count; }
+};
+struct AdvVarOp {
+    static constexpr int NS = 1;
+    const float* adv;
+    bool vec;
+    using Quad = float4;
+    __device__ bool aligned16() const { return vec; }
+    __device__ Quad load4(long long q) const { return reinterpret_cast<const float4*>(adv)[q]; }
+    __device__ static void one(float a, double mean, double* acc) { const double d = (double)a - mean; acc[0] += d * d; }
+    __device__ void add4(const Quad& g, double* acc) const
+    {
+        const double m = g_adv_stats[0];
+        one(g.x, m, acc); one(g.y, m, acc); one(g.z, m, acc); one(g.w, m, acc);
+    }
+    __device__ void add1(long long i, double* acc) const { one(adv[i], g_adv_stats[0], acc); }
+    __device__ void finish(const double* tot, long long count) const { g_adv_stats[1] = 1.0 / (sqrt(tot[0] / (double)count) + 1e-8); }
+};
+
+struct PpoOp {
+    static constexpr int NS = 4;
+    const float *logp_new, *logp_old, *values, *entropy, *adv, *returns;
+    float* out;
+    double clip;
+    bool normalize, vec;
+    struct Quad { float4 ln, lo, v, h, a, r; };
+    __device__ bool aligned16() const { return vec; }
+    __device__ Quad load4(long long q) const
+    {
+        return Quad{reinterpret_cast<const float4*>(logp_new)[q], reinterpret_cast<const float4*>(logp_old)[q],
+                    reinterpret_cast<const float4*>(values)[q], reinterpret_cast<const float4*>(entropy)[q],
+                    reinterpret_cast<const float4*>(adv)[q], reinterpret_cast<const float4*>(returns)[q]};
+    }
+    __device__ void one(float ln, float lo, float v, float h, float a, float r, double mean, double inv_std, double* acc) const
+    {
+        const double rho = exp((double)ln - (double)lo);
+        const double adv_n = ((double)a - mean) * inv_std;
+        const double clipped = fmin(fmax(rho, 1.0 - clip), 1.0 + clip);
+        acc[0] += fmin(rho * adv_n, clipped * adv_n);
+        const double d = (double)r - v;
+        acc[1] += d * d;
+        acc[2] += (double)h;
+        acc[3] += fabs(rho - 1.0) > clip ? 1.0 : 0.0;
+    }
+    __device__ void add4(const Quad& g, double* acc) const
+    {
+        const double m = normalize ? g_adv_stats[0] : 0.0, is = normalize ? g_adv_stats[1] : 1.0;
+        one(g.ln.x, g.lo.x, g.v.x, g.h.x, g.a.x, g.r.x, m, is, acc); one(g.ln.y, g.lo.y, g.v.y, g.h.y, g.a.y, g.r.y, m, is, acc);
+        one(g.ln.z, g.lo.z, g.v.z, g.h.z, g.a.z, g.r.z, m, is, acc); one(g.ln.w, g.lo.w, g.v.w, g.h.w, g.a.w, g.r.w, m, is, acc);
+    }
+    __device__ void add1(long long i, double* acc) const
+    {
+        const double m = normalize ? g_adv_stats[0] : 0.0, is = normalize ? g_adv_stats[1] : 1.0;
+        one(logp_new[i], logp_old[i], values[i], entropy[i], adv[i], returns[i], m, is, acc);
+    }
+    __device__ void finish(const double* tot, long long count) const
+    {
+        const double inv = 1.0 / (double)count;
+        for (int k = 0; k < 4; ++k) out[k] = (float)(tot[k] * inv);
+    }
+};
 
 }  // namespace
 }  // namespace hts
@@ -104,15 +228,28 @@ extern "C" hts_status hts_a2c_terms(const float* logp, const float* values, cons
 {
     using namespace hts;
     if (!logp || !values || !entropy || !returns || !out3 || count < 1) return HTS_ERR_INVALID_ARG;
-    long long blocks = (count + (long long)kThreads * kPerThread - 1) / ((long long)kThreads * kPerThread);
-    if (blocks > kBlocksMax) blocks = kBlocksMax;
-    long long per_block = (count + blocks - 1) / blocks;
-    per_block = (per_block + 3) / 4 * 4;
-    blocks = (count + per_block - 1) / per_block;
-    a2c_terms_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        logp, values, entropy, returns, (long long)count, per_block, out3);
-    HTS_LAUNCH_CHECK("a2c_terms_kernel");
-    return HTS_OK;
+    const A2cOp op{logp, values, entropy, returns, out3, all_aligned16({logp, values, entropy, returns})};
+    return launch_sums(op, (long long)count, static_cast<cudaStream_t>(cuda_stream), "a2c_terms");
+}
+
+extern "C" hts_status hts_ppo_terms(const float* logp_new, const float* logp_old, const float* values, const float* entropy,
+                                    const float* advantages, const float* returns, int64_t count, float clip,
+                                    int32_t normalize_advantages, float* out4, void* cuda_stream)
+{
+    using namespace hts;
+    if (!logp_new || !logp_old || !values || !entropy || !advantages || !returns || !out4 || count < 1) return HTS_ERR_INVALID_ARG;
+    if (!(clip > 0.f) || std::isinf(clip)) return HTS_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (normalize_advantages) {
+        const bool av = all_aligned16({advantages});
+        hts_status st = launch_sums(AdvMeanOp{advantages, av}, (long long)count, s, "adv_mean");
+        if (st != HTS_OK) return st;
+        st = launch_sums(AdvVarOp{advantages, av}, (long long)count, s, "adv_var");
+        if (st != HTS_OK) return st;
+    }
+    const PpoOp op{logp_new, logp_old, values, entropy, advantages, returns, out4, (double)clip, normalize_advantages != 0,
+                   all_aligned16({logp_new, logp_old, values, entropy, advantages, returns})};
+    return launch_sums(op, (long long)count, s, "ppo_terms");
 }
 
 // ---- the learner's parameter update (Section 4.1 "Delayed gradient", Eq. 5) ---------------------------------

@@ -193,3 +193,70 @@ def test_delayed_update_golden_and_refusals():
     assert L.hts_delayed_update(8, 16, 24, 4, 0.1, 1.5, 1e-5, None, None) == 1
     assert L.hts_delayed_update(8, 16, 24, 4, 0.1, 0.9, 0.0, None, None) == 1
     assert L.hts_delayed_update(8, 16, 24, 4, float("nan"), 0.9, 1e-5, None, None) == 1
+
+
+def gpu_ppo(ln, lo, v, h, a, r, clip, normalize):
+    t = [torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda() for x in (ln, lo, v, h, a, r)]
+    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    hts.hts_ppo_terms(*t, t[0].numel(), clip, normalize, out)
+    torch.cuda.synchronize()
+    return out.cpu().numpy()
+
+
+def test_ppo_terms_worked_example_on_gpu():
+    path = os.path.join(os.path.dirname(GOLD), "ppo_terms_worked_example.txt")
+    rows, exp = [], None
+    for line in open(path, encoding="utf-8"):
+        line = line.split("#")[0].strip()
+        if line.startswith("expected"):
+            exp = np.array([float(x) for x in line.split()[1:]])
+        elif line:
+            rows.append([float(x) for x in line.split()])
+    a = np.array(rows)
+    lo = np.full(len(a), -1.5, dtype=np.float32)
+    ln = (lo.astype(np.float64) + np.log(a[:, 0])).astype(np.float32)
+    got = gpu_ppo(ln, lo, a[:, 2], a[:, 4], a[:, 1], a[:, 3], 0.25, False)
+    assert np.allclose(got, exp, rtol=2e-6, atol=0)
+
+
+@pytest.mark.parametrize("count,normalize", [(1, False), (7, True), (4097, False), (4097, True), (131072, True),
+                                             ((1 << 21) + 5, True), (3000001, False)])
+def test_ppo_terms_against_oracle(count, normalize):
+    g = np.random.default_rng(count + int(normalize))
+    lo = (-g.random(count, dtype=np.float32) * 3).astype(np.float32)
+    ln = (lo + 0.25 * g.standard_normal(count, dtype=np.float32)).astype(np.float32)
+    v, r = g.standard_normal(count, dtype=np.float32), g.standard_normal(count, dtype=np.float32)
+    h = g.random(count, dtype=np.float32) * 2.8
+    adv = (1.5 * g.standard_normal(count, dtype=np.float32) + 0.7).astype(np.float32)
+    if count == 1:
+        normalize = False
+    got = gpu_ppo(ln, lo, v, h, adv, r, 0.2, normalize)
+    if count <= 200000:
+        ref = np.array(orc.ppo_terms(ln, lo, v, h, adv, r, 0.2, normalize))
+    else:                                               # the definition through fp64 library expressions at size
+        a64 = adv.astype(np.float64)
+        if normalize:
+            a64 = (a64 - a64.mean()) / (a64.std() + 1e-8)
+        rho = np.exp(ln.astype(np.float64) - lo)
+        ref = np.array([np.mean(np.minimum(rho * a64, np.clip(rho, 0.8, 1.2) * a64)),
+                        np.mean((r.astype(np.float64) - v) ** 2), np.mean(h, dtype=np.float64),
+                        np.mean(np.abs(rho - 1.0) > 0.2)])
+    floor = np.array([1.0 / np.sqrt(count), 1.0, 1.0, 1e-3])
+    # a sample whose |rho - 1| sits within rounding of the clip may fall on either side: one count of slack there
+    tol = 1e-6 * np.maximum(np.abs(ref), floor) + np.array([0, 0, 0, 2.0 / count])
+    assert np.all(np.abs(got - ref) <= tol), (got, ref)
+    assert np.array_equal(got, gpu_ppo(ln, lo, v, h, adv, r, 0.2, normalize))
+
+
+def test_ppo_terms_refusals_and_interleaving_with_a2c_terms():
+    L = hts.lib()
+    assert L.hts_ppo_terms(8, 16, 24, 32, 40, 48, 0, 0.2, 0, 56, None) == 1
+    assert L.hts_ppo_terms(8, 16, 24, 32, 40, 48, 4, 0.0, 0, 56, None) == 1
+    assert L.hts_ppo_terms(None, 16, 24, 32, 40, 48, 4, 0.2, 0, 56, None) == 1
+    # the two reductions share the library's partial table: back-to-back calls on one stream must not disturb each other
+    g = np.random.default_rng(0)
+    n = 50001
+    arrs = [g.standard_normal(n, dtype=np.float32) for _ in range(6)]
+    p1 = gpu_ppo(*arrs, 0.2, True)
+    a1 = gpu_terms(arrs[0], arrs[2], arrs[3], arrs[5])
+    assert np.array_equal(p1, gpu_ppo(*arrs, 0.2, True)) and np.array_equal(a1, gpu_terms(arrs[0], arrs[2], arrs[3], arrs[5]))
