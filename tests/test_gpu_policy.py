@@ -131,6 +131,26 @@ def test_other_frame_shapes(C, H, W, n):
         pol.close()
 
 
+@pytest.mark.parametrize("A,dtype", [(1, "bf16"), (64, "bf16"), (1, "fp32"), (64, "fp32"), (33, "bf16")])
+def test_extreme_action_counts(A, dtype):
+    """One action (the sampler has no choice, entropy 0) and the largest head the library takes."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS[2], A=A, weight_dtype=dtype)
+    n = 21
+    pol = Policy(cfg, max_batch=n)
+    try:
+        obs = wl.make_obs(cfg, n, batch_index=A)
+        ids = np.arange(70, 70 + n, dtype=np.int32)
+        got = pol.step(obs, ids, 4, 555)
+        ref = orc.policy_step(orc.Weights(pol.params), obs, ids, 4, 555)
+        check_against_oracle(cfg, got, ref, TOL[dtype])
+        check_sampler_on_gpu_logits(cfg, got, ids, np.full(n, 4), 555)
+        if A == 1:
+            assert np.all(got["actions"] == 0) and np.all(got["logp"] == 0.0) and np.all(got["entropy"] == 0.0)
+    finally:
+        pol.close()
+
+
 def test_uniform_stream_is_bit_exact():
     n, A, seed = 777, 19, 0xFEDCBA9876543210
     g = np.random.default_rng(0)
