@@ -478,6 +478,20 @@ def run_ours(args) -> None:
         tf5 = 2.0 * macs_per_env_step(c5) * nb / (us5 * 1e-6) / 1e12
         big = {"workload": c5.name, "n": nb, "us_per_step": us5, "env_steps_per_s": nb / (us5 * 1e-6), "tflops": tf5,
                "frac_of_bf16_sustained": tf5 / peak_tf, "frac_of_bf16_burst": tf5 / peaks["bf16_tflops"]}
+        # the same pool served as the asynchronous executors would hand it over: a random permutation cut into
+        # batches of random size 1..4096, each gathered from the state buffer and scattered into the storage row
+        batches = [torch.from_numpy(b).to(dev) for b in wl.make_async_batches(c5, nb, 4096)]
+        def serve(t):
+            for b in batches:
+                hts.hts_policy_step_indexed(ctx5, obs5[t % 2], nb, b, b, None, t, SEED, b.numel(), *o5, h_act_stream)
+        serve(0)
+        a5.record(s_act)
+        for t in range(10):
+            serve(t)
+        b5.record(s_act); torch.cuda.synchronize()
+        us_async = 1e3 * a5.elapsed_time(b5) / 10
+        big["async_batches"] = {"batches": len(batches), "sizes": [int(b.numel()) for b in batches],
+                                "us_per_pool_step": us_async, "env_steps_per_s": nb / (us_async * 1e-6)}
         hts.hts_policy_destroy(ctx5)
         del obs5
 
