@@ -173,6 +173,29 @@ def run_ncu_case(steps: int) -> None:
 
 
 # ------------------------------------------------------------------------------------------------
+def run_ncu_learner_case() -> None:
+    """The HBM-bound kernels on a shape larger than L2 but small enough to capture (2^25 transitions, 134 MB per
+    array, under 1.5 GB on the device): the advantage scan, both sample-mean kernels and the parameter update,
+    launched twice each (the second launch is the one to capture)."""
+    import torch
+    import paper_2012_09849_b200 as hts
+    cfg = wl.CONFIGS[WORKLOAD]
+    T, N = cfg.T, (1 << 25) // cfg.T
+    r, v, d, b = (torch.from_numpy(x).cuda() for x in wl.make_rollout(cfg, T=T, N=N))
+    adv, ret = torch.empty_like(v), torch.empty_like(v)
+    lp_new, lp_old = -torch.rand_like(v), -torch.rand_like(v)
+    out = torch.empty(4, device="cuda")
+    half = torch.empty(T * N, dtype=torch.bfloat16, device="cuda")
+    for _ in range(2):
+        hts.hts_gae(r, v, d, b, cfg.gamma, cfg.lam, T, N, adv, ret)
+        hts.hts_a2c_terms(lp_new, v, lp_old, ret, T * N, out)
+        hts.hts_ppo_terms(lp_new, lp_old, v, r, adv, ret, T * N, 0.2, True, out)
+        hts.hts_delayed_update(lp_new, adv, lp_old.abs_(), T * N, 7e-4, 0.99, 1e-5, half)
+    torch.cuda.synchronize()
+    print("ncu learner case done:", T * N, "transitions")
+
+
+# ------------------------------------------------------------------------------------------------
 def run_batch_sweep() -> None:
     """Actor-step time against the executor batch size, 1..8192 rows of the 8192-environment pool of the
     asynchronous-executor configuration (4x84x84 frames, 18 actions); prints a markdown table."""
@@ -563,9 +586,14 @@ def main():
                          "(no timing; for use under ncu)")
     ap.add_argument("--batch-sweep", action="store_true",
                     help="print actor-step time against the batch size (1..8192) and exit")
+    ap.add_argument("--ncu-learner-case", action="store_true",
+                    help="profiling driver: the HBM-bound kernels (advantage scan, sample means, update) on 2^25 "
+                         "transitions, twice each, and exit")
     args = ap.parse_args()
     if args.batch_sweep:
         run_batch_sweep()
+    elif args.ncu_learner_case:
+        run_ncu_learner_case()
     elif args.ncu_case > 0:
         run_ncu_case(args.ncu_case)
     elif args.impl == "reference":
