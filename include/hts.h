@@ -159,7 +159,7 @@ hts_status hts_a2c_terms(const float *logp, const float *values, const float *en
 
 /* The same for proximal policy optimisation, the algorithm HTS-RL is run with on the
  * football scenarios (Section 5, "Ours (PPO)"; objective of Schulman et al. 2017, Eq. 7):
- *   rho_i   = exp(logp_new_i - logp_old_i)
+ *   rho_i   = exp(logp_new_i - logp_old_i)   (fp32 exponential; everything after it in fp64)
  *   A_i     = advantages_i, or (advantages_i - mean) / (std + 1e-8) over the batch
  *             (population std) if normalize_advantages != 0
  *   out4[0] = (1/count) sum min(rho_i A_i, clip(rho_i, 1-clip, 1+clip) A_i)   clipped surrogate

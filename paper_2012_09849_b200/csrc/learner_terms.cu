@@ -193,7 +193,7 @@ struct PpoOp {
     }
     __device__ void one(float ln, float lo, float v, float h, float a, float r, double mean, double inv_std, double* acc) const
     {
-        const double rho = exp((double)ln - (double)lo);
+        const double rho = (double)expf(ln - lo);           // fp32 exponential (2 ulp): the fp64 one would bound the kernel
         const double adv_n = ((double)a - mean) * inv_std;
         const double clipped = fmin(fmax(rho, 1.0 - clip), 1.0 + clip);
         acc[0] += fmin(rho * adv_n, clipped * adv_n);
