@@ -22,6 +22,9 @@
  *   - Calls taking a `cuda_stream` (a cudaStream_t passed as void*, NULL = legacy
  *     default stream) only enqueue work on that stream and do not synchronise.
  *   - Output buffers must not overlap input buffers or each other.
+ *   - A context owns one activation workspace: its steps must be ordered on the GPU
+ *     (one stream, or events between streams).  Steps that may overlap need a
+ *     context each; contexts are independent, also across threads.
  *   - There is no CPU fallback: without a CUDA device calls return HTS_ERR_CUDA.
  */
 #ifndef HTS_H_
