@@ -232,6 +232,15 @@ const char *hts_policy_kernel_name(int32_t kernel);
  * nothing was recorded.  Synchronises with the device.                            */
 hts_status hts_last_async_error(hts_ctx *ctx);
 
+/* Self-test of the failure-detection path (the kernels of this library never wait
+ * without a limit: a pipeline stage that does not get its data within about a second
+ * records a code, the block drains and the kernel returns, and hts_last_async_error
+ * reports HTS_ERR_TIMEOUT).  This call enqueues one tiny block that waits, through the
+ * same helper, on a barrier nothing arrives on, gives up after `limit_ticks` SM clock
+ * ticks (1e3 .. 1e8) and returns normally; afterwards hts_last_async_error(ctx) must
+ * report HTS_ERR_TIMEOUT once and the context must still work.  Errors: INVALID_ARG, CUDA. */
+hts_status hts_wait_selftest(hts_ctx *ctx, int64_t limit_ticks, void *cuda_stream);
+
 void hts_policy_destroy(hts_ctx *ctx);
 
 /* Advantages and returns over the rollout storage (Section 3: with lambda = 1,

@@ -26,7 +26,7 @@ EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "h
            "hts_policy_evaluate", "hts_a2c_terms", "hts_ppo_terms", "hts_delayed_update",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
-           "hts_gae_host", "hts_policy_step_noalloc", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
+           "hts_gae_host", "hts_policy_step_noalloc", "hts_wait_selftest", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
 
 
 class HtsError(RuntimeError):
@@ -85,6 +85,8 @@ def lib():
         L.hts_policy_kernel_name.argtypes = [i32]
         L.hts_policy_kernel_name.restype = C.c_char_p
         L.hts_last_async_error.argtypes = [vp]
+        L.hts_wait_selftest.argtypes = [vp, C.c_int64, vp]
+        L.hts_wait_selftest.restype = C.c_int
         L.hts_policy_destroy.argtypes = [vp]
         L.hts_policy_destroy.restype = None
         gae = [vp, vp, vp, vp, f32, f32, i32, i32, vp, vp, vp]
@@ -211,6 +213,10 @@ def hts_policy_kernel_name(kernel: int) -> str:
 
 def hts_last_async_error(ctx) -> int:
     return int(lib().hts_last_async_error(ctx))
+
+
+def hts_wait_selftest(ctx, limit_ticks: int, stream=None) -> None:
+    _check(lib().hts_wait_selftest(ctx, int(limit_ticks), _stream(stream)), "hts_wait_selftest")
 
 
 def hts_policy_destroy(ctx) -> None:

@@ -93,7 +93,7 @@ struct Profiler {
     void end(int k, cudaStream_t s) { if (on && used[k] < kCap) { cudaEventRecord(stop[k][used[k]], s); ++used[k]; } }
 };
 
-// ---- the fp32 CUDA-core path (check path; also the fallback arithmetic for bf16 weights) ---
+// ---- the fp32 CUDA-core path (the check path for fp32 weights; bf16 contexts never use it) ---
 struct RefWeights {            // fp32 device copies in PyTorch layouts
     float *w1, *b1, *w2, *b2, *w3, *b3, *wfc, *bfc;
     float *whead, *bhead;      // [A+1,512], [A+1]: policy rows then the value row
@@ -131,6 +131,9 @@ hts_status launch_heads(const float* h_partials, int num_splits, size_t split_st
 
 hts_status launch_uniforms(const int32_t* env_ids, const int32_t* t_per_env, int32_t t, uint64_t seed, int n,
                            int A, float* out, cudaStream_t s);
+
+// ---- self-test of the bounded wait (reports through the status word like any expired wait) ---
+hts_status launch_wait_selftest(long long limit_ticks, int* status, cudaStream_t s);
 
 // ---- advantage scan -------------------------------------------------------------------------
 hts_status launch_gae(const float* rewards, const float* values, const uint8_t* dones,

@@ -80,10 +80,14 @@ bool any_overlap(const Range* in, int nin, const Range* out, int nout)
 }
 
 hts_status check_step_args(hts_ctx* ctx, const void* obs, const void* env_ids, int n,
-                           const void* actions, const void* logp, const void* values, const void* entropy)
+                           const void* actions, const void* logp, const void* values, const void* entropy,
+                           bool on_host = false)
 {
     if (!ctx || !obs || !env_ids || !actions || !logp || !values || !entropy) return HTS_ERR_INVALID_ARG;
     if (n < 1 || n > ctx->desc.max_batch) return HTS_ERR_INVALID_ARG;
+    // the tensor-core path stages frames with bulk copies, which need 16-byte-aligned global addresses
+    // (frame, channel and row-group offsets are multiples of 16 because H and W are multiples of 4)
+    if (ctx->tc && !on_host && ((uintptr_t)obs & 15u) != 0) return HTS_ERR_INVALID_ARG;
     if (!ctx->loaded) return HTS_ERR_UNSUPPORTED;
     return HTS_OK;
 }
@@ -221,6 +225,7 @@ hts_status hts_policy_evaluate(hts_ctx* ctx, const uint8_t* obs, const int32_t* 
 {
     if (!ctx || !obs || !actions || !logp || !values || !entropy) return HTS_ERR_INVALID_ARG;
     if (n < 1 || n > ctx->desc.max_batch) return HTS_ERR_INVALID_ARG;
+    if (ctx->tc && ((uintptr_t)obs & 15u) != 0) return HTS_ERR_INVALID_ARG;
     if (!ctx->loaded) return HTS_ERR_UNSUPPORTED;
     const size_t nn = (size_t)n;
     const Range in[] = {{obs, nn * ctx->g.C * ctx->g.H * ctx->g.W}, {actions, nn * 4}};
@@ -235,7 +240,7 @@ hts_status hts_policy_step_host(hts_ctx* ctx, const uint8_t* obs, const int32_t*
                                 int32_t* actions, float* logp, float* values, float* entropy,
                                 float* logits_or_null, void* cuda_stream)
 {
-    hts_status st = check_step_args(ctx, obs, env_ids, n, actions, logp, values, entropy);
+    hts_status st = check_step_args(ctx, obs, env_ids, n, actions, logp, values, entropy, true);
     if (st != HTS_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t nn = (size_t)n;
@@ -286,6 +291,12 @@ hts_status hts_last_async_error(hts_ctx* ctx)
         return (word == kStatusBadSlot || word == kStatusBadAction) ? HTS_ERR_INVALID_ARG : HTS_ERR_TIMEOUT;
     }
     return HTS_OK;
+}
+
+hts_status hts_wait_selftest(hts_ctx* ctx, int64_t limit_ticks, void* cuda_stream)
+{
+    if (!ctx || limit_ticks < 1000 || limit_ticks > 100000000LL) return HTS_ERR_INVALID_ARG;
+    return launch_wait_selftest((long long)limit_ticks, ctx->status, static_cast<cudaStream_t>(cuda_stream));
 }
 
 hts_status hts_policy_profile(hts_ctx* ctx, int32_t enable)

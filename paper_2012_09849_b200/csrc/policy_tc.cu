@@ -35,7 +35,7 @@ constexpr int BM = 128;                 // rows per tile = TMEM lanes
 constexpr int BK = 64;                  // 16-bit elements per K chunk = one 128-byte swizzle row
 constexpr int STAGES = 3;                 // 3 x 32 KiB: two CTAs per SM, so the 224 FC tiles run in one wave
 constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
-enum { EPI_CONV = 0, EPI_SPLITK = 1 };
+enum { EPI_SPLITK = 1 };
 enum { L_CONV1 = 0, L_CONV2, L_CONV3, L_FC, L_COUNT };
 
 struct GemmParams {
@@ -136,7 +136,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (ok) {
             const long m = (long)m0 + r;
             const float inv = *p.inv_scale;
-            if (EPI == EPI_SPLITK) {
+            {
                 // The accumulator arrives one row per thread; a row-per-thread store would touch 32
                 // lines per instruction.  Each warp turns its 32x32 block through shared memory (the
                 // pipeline stages are free by now) so that eight lanes write one full 128-byte line.
@@ -161,29 +161,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (m0 + q * 32 + rr < p.n_env) *reinterpret_cast<float4*>(dst + (size_t)rr * p.ldo + c + c4) = val;
                     }
                     __syncwarp();
-                }
-            } else {
-                const int env = (int)(m / p.P_in);
-                const int pix = (int)(m - (long)env * p.P_in);
-                const int y = pix / p.W_in, x = pix - y * p.W_in;
-                const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
-                __half* dst = p.out_h + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * BN;
-#pragma unroll
-                for (int c = 0; c < BN; c += 32) {
-                    uint32_t v[32];
-                    tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
-                    tmem_ld_wait();
-                    if (valid) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int h = 0; h < 4; ++h)
-                                pk[h] = pack_relu_h2(fmaf(__uint_as_float(v[j + 2 * h]), inv, p.bias[n0 + c + j + 2 * h]),
-                                                     fmaf(__uint_as_float(v[j + 2 * h + 1]), inv, p.bias[n0 + c + j + 2 * h + 1]));
-                            *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        }
-                    }
                 }
             }
         }
@@ -321,7 +298,7 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     if (!t) return HTS_ERR_ALLOC;
     t->g = g; t->max_batch = max_batch; t->status = status;
     if (!conv1_plan(g, &t->pl1)) { delete t; return HTS_ERR_SHAPE; }
-    t->H1s = (g.H1 + 1) / 2; t->W1s = (g.W1 + 1) / 2; t->P1s = t->H1s * t->W1s;
+    t->H1s = t->pl1.H1s; t->W1s = t->pl1.W1s; t->P1s = t->pl1.P1s;
     t->P2 = g.H2 * g.W2; t->P3 = g.H3 * g.W3;
     const int chunks = g.F / BK;
     t->splits = 1;
@@ -330,7 +307,7 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     const size_t nb = (size_t)max_batch;
     auto A = [&](auto** p, size_t count) { return alloc(alloc_ctx, reinterpret_cast<void**>(p), count * sizeof(**p)); };
     bool ok = A(&t->w2p, (size_t)64 * 512) && A(&t->w3p, (size_t)64 * 576) && A(&t->wfcp, (size_t)512 * g.F) &&
-              A(&t->w1p, (size_t)32 * 4 * t->pl1.Cs) && A(&t->b1, 32) && A(&t->b2, 64) && A(&t->b3, 64) && A(&t->bfc, 512) &&
+              A(&t->w1p, (size_t)128 * 16 * g.C) && A(&t->b1, 32) && A(&t->b2, 64) && A(&t->b3, 64) && A(&t->bfc, 512) &&
               A(&t->whead, (size_t)(g.A + 1) * 512) && A(&t->bhead, (size_t)g.A + 1) &&
               A(&t->absmax, L_COUNT) && A(&t->scale, L_COUNT) && A(&t->inv_scale, L_COUNT) &&
               A(&t->a1s, nb * t->P1s * 128) && A(&t->a2, nb * t->P2 * 64) && A(&t->a3, nb * g.F) &&
@@ -341,7 +318,7 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
     t->rows2 = conv_res_tile_rows(t->W1s + 1);
     t->rows3 = conv_res_tile_rows(2 * g.W2 + 2);
     if (t->rows2 > 256 || t->rows3 > 256) { delete t; return HTS_ERR_SHAPE; }
-    ok = make_map(&t->mW1, t->w1p, 32, 4 * t->pl1.Cs, (uint64_t)8 * t->pl1.Cs, 32) &&
+    ok = make_map(&t->mW1, t->w1p, 128, 16 * g.C, (uint64_t)32 * g.C, 64) &&
          make_map(&t->mA2, t->a1s, nb * t->P1s, 128, 256, t->rows2) && make_map(&t->mB2, t->w2p, 64, 512, 1024, 64) &&
          make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, t->rows3) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
          make_map(&t->mAfc, t->a3, nb, g.F, (uint64_t)g.F * 2, BM) && make_map(&t->mBfc, t->wfcp, 512, g.F, (uint64_t)g.F * 2, 128);

@@ -40,7 +40,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 // Failed polls back off with a short sleep: polling threads read shared memory, and the tensor
 // core fetches its operands from the same shared memory.
 constexpr long long kWaitLimitTicks = 2000000000LL;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                          long long limit_ticks = kWaitLimitTicks)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -49,7 +50,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((spins & 63) == 63) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitTicks) {
+            if (clock64() - t0 > limit_ticks) {
                 *abort_flag = 1;
                 if (status) atomicCAS(status, 0, code);
                 return false;
