@@ -17,24 +17,36 @@
 //     ReLU and stores fp16 in the layout conv2 reads.  Warp quarters overlap by one lane (quarter k
 //     starts at column 31 k of the tile), so the neighbour is always in the same warp.
 //
-// Work unit = (tile of 125 grid columns, range of output rows).  A CTA is a pipeline of four roles:
-// warp 0 stages the four input rows under a grid row (one bulk copy per environment and channel)
-// into a ring in shared memory; warps 4..7 convert (thread = grid column) and write tensor memory;
-// lane 0 of warps 1 and 2 issue the MMAs of alternate steps, each into its own accumulator; warps
-// 8..11 run the epilogue.  All waits are bounded.
+// Work unit = (tile of 125 grid columns, range of output rows).  One CTA per SM runs a pipeline of
+// four roles.  One thread stages groups of grid rows into a ring in shared memory: one tensor-tiled
+// TMA box per environment (all channels, group_rows x 4 input rows; the frames are viewed as 32-bit
+// words so that a box row is the 4 W contiguous bytes under one grid row).  Two groups of four
+// converter warps take alternate grid rows (thread = grid column), expand them in registers and write
+// tensor memory; two threads issue the MMAs of alternate steps, each step into the next of several
+// accumulators; two groups of four epilogue warps drain alternate steps.  Every role is bound by
+// latency chains (shared -> registers -> tensor memory, tensor memory -> registers -> global), which
+// is why each exists twice.  All waits are bounded.
 #include "conv1_tc.cuh"
 #include "tc_ptx.cuh"
+#include "tc_host.cuh"
 
 namespace hts {
 using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 384;                   // warp 0 copies, 1 and 2 issue, 3 idle, 4..7 convert, 8..11 epilogue
+#ifndef HTS_CONV1_ISSUERS
+#define HTS_CONV1_ISSUERS 4
+#endif
+constexpr int kIssuers = HTS_CONV1_ISSUERS;     // one thread issues an MMA every 60 clocks or so; a 128 x 64 x 16 one runs for 32
+constexpr int kConvWarp0 = kIssuers + 1;        // warp 0 stages, 1..kIssuers issue, then 8 converter and 8 epilogue warps
+constexpr int kEpiWarp0 = kConvWarp0 + 8;
+constexpr int kThreads = (kEpiWarp0 + 8) * 32;
 constexpr int kTileCols = 124;                  // new grid columns per tile (4 quarters x 31; one more is shared)
 constexpr int kChunkBytes = 64 * 128;           // one filter K chunk: 64 rows (dx, o) x 64 fp16
 constexpr int kMaxStages = 8;
-constexpr int kMaxRing = 4;
+constexpr int kMaxRing = 8;
+constexpr int kMaxAcc = 4;
 
 struct Conv1Params {
     Conv1Plan pl;
@@ -43,7 +55,8 @@ struct Conv1Params {
     int pool;               // frames in obs when slots are given
     int n;
     int tiles;              // ceil(n * Ws / 124)
-    int splits;             // ranges the H1 output rows of a tile are cut into
+    int splits;             // equal ranges the H1 output rows of a tile are cut into (a divisor of H1)
+    int su;                 // output rows (steps) per unit: H1 / splits; a unit stages su + 1 grid rows
     const float* bias;
     const float* inv_scale;
     __half* out;
@@ -76,30 +89,55 @@ __device__ __forceinline__ uint32_t relu_pack_h2(float lo, float hi)
     return r;
 }
 
-// the unit's tile and output-row range
-struct Unit {
-    int tile, y0, y1;
-    __device__ __forceinline__ void set(int u, int splits, int H1)
+// Position of a role in the CTA's sequence of units.  The CTA's units are u = blockIdx.x + i * gridDim.x; every
+// unit has `su` steps (output rows) and su + 1 grid rows, so a role that takes every k-th step or row of the
+// CTA's sequence finds its unit by stepping a counter instead of dividing.
+struct Walk {
+    int i, pos;                 // unit of this CTA, position inside it (step or row)
+    int tile, y_base;           // the unit's tile and first output row
+    __device__ __forceinline__ void unit(const Conv1Params& p)
     {
-        tile = u / splits;
-        const int part = u - tile * splits;
-        y0 = part * H1 / splits;
-        y1 = (part + 1) * H1 / splits;
+        const int u = blockIdx.x + i * gridDim.x;
+        tile = u / p.splits;
+        y_base = (u - tile * p.splits) * p.su;
+    }
+    __device__ __forceinline__ void start(const Conv1Params& p, int first) { i = 0; pos = first; }
+    // brings pos back below `len` (items per unit); true if the unit changed
+    __device__ __forceinline__ bool settle(int len)
+    {
+        bool moved = false;
+        while (pos >= len) { pos -= len; ++i; moved = true; }
+        return moved;
     }
 };
 
+// packed fp32 pairs (sm_100): two lanes of an add / fused multiply-add per instruction
+__device__ __forceinline__ void add2(float& a0, float& a1, float b0, float b1)
+{
+    asm("{\n\t.reg .b64 ra, rb;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
+        "add.rn.f32x2 ra, ra, rb;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fma2(float& a0, float& a1, float m, float c0, float c1)
+{
+    asm("{\n\t.reg .b64 ra, rm, rc;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rm, {%2, %2};\n\tmov.b64 rc, {%3, %4};\n\t"
+        "fma.rn.f32x2 ra, ra, rm, rc;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(m), "f"(c0), "f"(c1));
+}
+
 // CG: groups of four channels.  WC: the frame width when known at compile time (the converter's loads then
-// use immediate offsets), 0 = any.  NI: issuing threads.
+// use immediate offsets), 0 = any.
 template <int CG, int WC>
-__global__ void __launch_bounds__(kThreads, CG == 1 ? 2 : 1)
-conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
+__global__ void __launch_bounds__(kThreads, 1)
+conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const Conv1Params p)
 {
     const Conv1Plan& pl = p.pl;
-    constexpr int C = 4 * CG;
     constexpr int ACOLS = 32 * CG;                     // tensor-memory columns of one operand row
+    constexpr int KR = CG == 1 ? 3 : 1;                // grid rows per staged group (= pl.group_rows)
+    constexpr int NACC = CG == 4 ? 2 : 4;              // accumulators (= pl.accs)
+    constexpr int R = CG == 1 ? 8 : CG == 2 ? 4 : 3;   // operand rows in the ring (= pl.ring)
     const int W = WC ? WC : pl.W;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t w_bar, u8_full[kMaxStages], u8_empty[kMaxStages], a_full[kMaxRing], a_empty[kMaxRing], d_full[2], d_empty[2];
+    __shared__ uint64_t w_bar, u8_full[kMaxStages], u8_empty[kMaxStages], a_full[kMaxRing], a_empty[kMaxRing],
+        d_full[kMaxAcc], d_empty[kMaxAcc];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ __align__(16) float s_bias[32];
@@ -109,25 +147,26 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     constexpr int w_bytes = 2 * CG * kChunkBytes;
     uint8_t* s_u8 = sm + w_bytes;
-    const int NS = pl.stages, R = pl.ring;
+    const int NS = pl.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int units = p.tiles * p.splits;
 
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 128); }
-        for (int s = 0; s < kMaxRing; ++s) { mbar_init(&a_full[s], 128); mbar_init(&a_empty[s], 2); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 128); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 8); }
+        for (int s = 0; s < kMaxRing; ++s) { mbar_init(&a_full[s], 4); mbar_init(&a_empty[s], 2); }
+        for (int s = 0; s < kMaxAcc; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 4); }
         abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmX);
     }
-    if (threadIdx.x >= 96 && threadIdx.x < 128) s_bias[threadIdx.x - 96] = p.bias[threadIdx.x - 96];
-    if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)pl.tmem_cols);
+    if (threadIdx.x >= 32 && threadIdx.x < 64) s_bias[threadIdx.x - 32] = p.bias[threadIdx.x - 32];
+    if (warp == 1) tmem_alloc(&tmem_slot, 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_d = tmem_slot, tmem_a = tmem_slot + 128;     // two accumulators of 64 columns, then the ring
+    const uint32_t tmem_d = tmem_slot, tmem_a = tmem_slot + NACC * 64;   // accumulators of 64 columns, then the ring
     if (threadIdx.x == 0) {                                   // the filter does not depend on the previous kernel
         mbar_arrive_expect_tx(&w_bar, (uint32_t)w_bytes);
         for (int dy = 0; dy < 2; ++dy)
@@ -136,163 +175,192 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     pdl_wait();
     pdl_trigger();
 
+    const int my_units = blockIdx.x < units ? (units - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const int su = p.su, ru = p.su + 1;                       // steps and grid rows per unit
+    const int total_steps = my_units * su;
+
     if (warp == 0) {
-        // ---- staging: the four input rows under grid row Y, for every environment the tile touches
-        const size_t chan = (size_t)pl.H * W, frame = chan * C;
-        const uint32_t row_bytes = 4u * (uint32_t)W;
-        int st = 0;
-        uint32_t stph = 0;
-        Unit un;
-        for (int u = blockIdx.x; u < units; u += gridDim.x) {
-            un.set(u, p.splits, pl.H1);
-            const int e_first = (un.tile * kTileCols) / pl.Ws;
-            int e_last = (un.tile * kTileCols + kTileCols) / pl.Ws;
-            if (e_last > p.n - 1) e_last = p.n - 1;
-            const int copies = (e_last - e_first + 1) * C;
+        // ---- staging: groups of KR grid rows, one box per environment the tile touches
+        if (lane == 0) {
+            int st = 0;
+            uint32_t stph = 0;
             bool alive = true;
-            for (int Y = un.y0; Y <= un.y1; ++Y) {
-                if (!mbar_wait_warp(&u8_empty[st], stph ^ 1u, abortp, p.status, 31)) { alive = false; break; }
-                uint8_t* dst = s_u8 + st * pl.stage_bytes;
-                if (lane == 0) mbar_arrive_expect_tx(&u8_full[st], (uint32_t)copies * row_bytes);
-                __syncwarp();
-                for (int i = lane; i < copies; i += 32) {
-                    const int ei = i / C, c = i - ei * C;
-                    const uint8_t* src = p.obs + frame_of(p, e_first + ei) * frame + c * chan + (size_t)(4 * Y) * W;
-                    bulk_load(dst + i * row_bytes, src, row_bytes, &u8_full[st]);
+            Walk w;
+            for (w.i = 0; alive && w.i < my_units; ++w.i) {
+                w.unit(p);
+                const int e_first = (w.tile * kTileCols) / pl.Ws;
+                int e_last = (w.tile * kTileCols + kTileCols) / pl.Ws;
+                if (e_last > p.n - 1) e_last = p.n - 1;
+                const int envs = e_last - e_first + 1;
+                for (int Y = w.y_base; Y <= w.y_base + su; Y += KR) {
+                    if (!mbar_wait(&u8_empty[st], stph ^ 1u, abortp, p.status, 31)) { alive = false; break; }
+                    uint8_t* dst = s_u8 + st * pl.stage_bytes;
+                    mbar_arrive_expect_tx(&u8_full[st], (uint32_t)(envs * pl.env_bytes));
+                    for (int i = 0; i < envs; ++i)
+                        tma_load_4d(dst + i * pl.env_pitch, &tmX, 0, Y, 0, (int)frame_of(p, e_first + i), &u8_full[st]);
+                    if (++st == NS) { st = 0; stph ^= 1u; }
                 }
-                if (++st == NS) { st = 0; stph ^= 1u; }
             }
-            if (!alive) break;
         }
-    } else if (warp == 1 || warp == 2) {
-        // ---- MMA issue: thread g takes the CTA's steps g, g + 2, ... into accumulator g
+    } else if (warp <= kIssuers) {
+        // ---- MMA issue: thread g takes the CTA's steps g, g + kIssuers, ...; step k goes to accumulator k % NACC.
+        //      Step k of the CTA reads operand rows k + (its unit's index) and the next one.
         if (lane == 0) {
             const int g = warp - 1;
             constexpr uint32_t idesc = instr_desc_f16(0, 128, 64);
+            uint64_t bdesc[2][CG];
+#pragma unroll
+            for (int dy = 0; dy < 2; ++dy)
+#pragma unroll
+                for (int cg = 0; cg < CG; ++cg) bdesc[dy][cg] = smem_desc_sw128(base + (dy * CG + cg) * kChunkBytes);
             bool alive = mbar_wait(&w_bar, 0, abortp, p.status, 32);
-            const uint32_t d_addr = tmem_d + g * 64;
-            int s = 0;                                    // ring entry of grid row Y = y and the parity of its current use
-            uint32_t sph = 0;
-            int sc = 0;                                   // steps of this CTA so far
-            Unit un;
-            for (int u = blockIdx.x; alive && u < units; u += gridDim.x) {
-                un.set(u, p.splits, pl.H1);
-                for (int y = un.y0; y < un.y1; ++y, ++sc) {
-                    const int s1 = s + 1 == R ? 0 : s + 1;
-                    const uint32_t ph1 = s + 1 == R ? sph ^ 1u : sph;
-                    if ((sc & 1) == g) {
-                        if (!mbar_wait(&d_empty[g], (((uint32_t)sc >> 1) & 1u) ^ 1u, abortp, p.status, 33)) { alive = false; break; }
-                        if (!mbar_wait(&a_full[s], sph, abortp, p.status, 34)) { alive = false; break; }
-                        if (!mbar_wait(&a_full[s1], ph1, abortp, p.status, 34)) { alive = false; break; }
-                        tc_fence_after();
+            Walk w;
+            w.start(p, g);
+            for (int k = g; alive && k < total_steps; k += kIssuers, w.pos += kIssuers) {
+                w.settle(su);
+                const int r0 = k + w.i, r1 = r0 + 1;                       // operand rows of this step
+                const int s0 = r0 % R, s1 = r1 % R;
+                const int acc = k % NACC;
+                if (!mbar_wait(&d_empty[acc], (((uint32_t)(k / NACC)) & 1u) ^ 1u, abortp, p.status, 33)) break;
+                if (!mbar_wait(&a_full[s0], ((uint32_t)(r0 / R)) & 1u, abortp, p.status, 34)) break;
+                if (!mbar_wait(&a_full[s1], ((uint32_t)(r1 / R)) & 1u, abortp, p.status, 34)) break;
+                tc_fence_after();
+                const uint32_t d_addr = tmem_d + acc * 64;
 #pragma unroll
-                        for (int dy = 0; dy < 2; ++dy) {
-                            const uint32_t a_addr = tmem_a + (dy ? s1 : s) * ACOLS;
+                for (int dy = 0; dy < 2; ++dy) {
+                    const uint32_t a_addr = tmem_a + (dy ? s1 : s0) * ACOLS;
 #pragma unroll
-                            for (int cg = 0; cg < CG; ++cg) {
-                                const uint64_t bdesc = smem_desc_sw128(base + (dy * CG + cg) * kChunkBytes);
+                    for (int cg = 0; cg < CG; ++cg)
 #pragma unroll
-                                for (int k = 0; k < 4; ++k)
-                                    mma_f16_ts(d_addr, a_addr + cg * 32 + 8 * k, bdesc + 2 * k, idesc, (dy | cg | k) != 0);
-                            }
-                        }
-                        // an operand row is read by two steps (as the lower and as the upper grid row); the first
-                        // and the last row of a unit by one only, which then arrives for both
-                        mma_commit(&a_empty[s]);
-                        mma_commit(&a_empty[s1]);
-                        if (y == un.y0) mma_commit(&a_empty[s]);
-                        if (y == un.y1 - 1) mma_commit(&a_empty[s1]);
-                        mma_commit(&d_full[g]);
-                    }
-                    s = s1; sph = ph1;
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_f16_ts(d_addr, a_addr + cg * 32 + 8 * kk, bdesc[dy][cg] + 2 * kk, idesc, (dy | cg | kk) != 0);
                 }
-                if (++s == R) { s = 0; sph ^= 1u; }       // past the unit's last grid row
+                mma_commit(&d_full[acc]);
             }
         }
-    } else if (warp >= 4 && warp < 8) {
-        // ---- convert: thread = grid column q of the tile, one operand row per staged grid row
+    } else if (warp < kEpiWarp0) {
+        // ---- convert: thread = grid column q of the tile; group h takes the CTA's grid rows h, h + 2, ...
+        const int h = (warp - kConvWarp0) >> 2;
         const int qq = warp & 3;
         const uint32_t st_addr = tmem_a + ((uint32_t)(qq * 32) << 16);
-        int s = 0, st = 0;
-        uint32_t sph = 0, stph = 0;
-        Unit un;
+        int st = 0;                                       // staged group
+        uint32_t stph = 0;
+        int r = 0;                                        // grid rows of this CTA so far
+        int pending = -1;                                 // ring entry whose tensor-memory stores are still in flight
         bool alive = true;
-        for (int u = blockIdx.x; alive && u < units; u += gridDim.x) {
-            un.set(u, p.splits, pl.H1);
-            const int q = un.tile * kTileCols + 31 * qq + lane;
+        Walk w;
+        for (w.i = 0; alive && w.i < my_units; ++w.i) {
+            w.unit(p);
+            const int q = w.tile * kTileCols + 31 * qq + lane;
             const int e = q / pl.Ws, X = q - e * pl.Ws;
-            const int e_first = (un.tile * kTileCols) / pl.Ws;
+            const int e_first = (w.tile * kTileCols) / pl.Ws;
             // columns past the end of the batch read the start of the buffer: their results are never stored
-            const int off = e < p.n ? (e - e_first) * C * 4 * W + 4 * X : 0;
-            for (int Y = un.y0; Y <= un.y1; ++Y) {
-                if (!mbar_wait_warp(&u8_full[st], stph, abortp, p.status, 35)) { alive = false; break; }
-                const uint8_t* src = s_u8 + st * pl.stage_bytes + off;
+            const int off = e < p.n ? (e - e_first) * pl.env_pitch + 4 * X : 0;
+            int yr = 0;                                   // row inside the staged group
+            for (int j = 0; j < ru; ++j, ++r) {
+                if (yr == 0 && !mbar_wait_warp(&u8_full[st], stph, abortp, p.status, 35)) { alive = false; break; }
+                if ((r & 1) == h) {
+                    const int s = r % R;
+                    const uint8_t* src = s_u8 + st * pl.stage_bytes + off + yr * 4 * W;
 #pragma unroll
-                for (int cg = 0; cg < CG; ++cg) {
-                    uint32_t r[32];
+                    for (int cg = 0; cg < CG; ++cg) {
+                        uint32_t v[32];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
+                        for (int c = 0; c < 4; ++c)
 #pragma unroll
-                        for (int uy = 0; uy < 4; ++uy)
-                            u8x4_to_h4(*reinterpret_cast<const uint32_t*>(src + ((cg * 4 + c) * 4 + uy) * W),
-                                       r[c * 8 + uy * 2], r[c * 8 + uy * 2 + 1]);
-                    if (cg == CG - 1) mbar_arrive(&u8_empty[st]);         // the staged rows are in registers
-                    if (cg == 0) {
-                        if (!mbar_wait_warp(&a_empty[s], sph ^ 1u, abortp, p.status, 36)) { alive = false; break; }
-                        tc_fence_after();
+                            for (int uy = 0; uy < 4; ++uy)
+                                u8x4_to_h4(*reinterpret_cast<const uint32_t*>(src + ((cg * 4 + c) * KR * 4 + uy) * W),
+                                           v[c * 8 + uy * 2], v[c * 8 + uy * 2 + 1]);
+                        if (cg == 0) {
+                            if (pending >= 0) {               // the previous row's stores overlapped these loads
+                                tmem_st_wait();
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&a_full[pending]);
+                            }
+                            if (!mbar_wait_warp(&a_empty[s], (((uint32_t)(r / R)) & 1u) ^ 1u, abortp, p.status, 36)) { alive = false; break; }
+                            tc_fence_after();
+                        }
+                        tmem_st_32x32(st_addr + s * ACOLS + cg * 32, v);
                     }
-                    tmem_st_32x32(st_addr + s * ACOLS + cg * 32, r);
+                    if (!alive) break;
+                    pending = s;
                 }
-                if (!alive) break;
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&a_full[s]);
-                if (++s == R) { s = 0; sph ^= 1u; }
-                if (++st == NS) { st = 0; stph ^= 1u; }
+                if (++yr == KR || j == ru - 1) {          // done with this staged group (every converter warp arrives)
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&u8_empty[st]);
+                    yr = 0;
+                    if (++st == NS) { st = 0; stph ^= 1u; }
+                }
             }
         }
-    } else if (warp >= 8) {
-        // ---- epilogue: warps 8..11 read TMEM lane quarters 0..3
+        if (pending >= 0) {
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[pending]);
+        }
+    } else {
+        // ---- epilogue: group g drains the CTA's steps g, g + 2, ...; warp quarter = TMEM lane quarter
+        const int g = (warp - kEpiWarp0) >> 2;
         const int qq = warp & 3;
         const float inv = *p.inv_scale;
-        int sc = 0;
-        Unit un;
-        bool alive = true;
-        for (int u = blockIdx.x; alive && u < units; u += gridDim.x) {
-            un.set(u, p.splits, pl.H1);
-            const int q = un.tile * kTileCols + 31 * qq + lane;
-            const int e = q / pl.Ws, X = q - e * pl.Ws;
-            const bool valid = lane < 31 && e < p.n && X < pl.W1;
-            __half* dst0 = p.out + ((size_t)e * pl.P1s + (X >> 1)) * 128 + (X & 1) * 32;
-            for (int y = un.y0; y < un.y1; ++y, ++sc) {
-                const int acc = sc & 1;
-                if (!mbar_wait_warp(&d_full[acc], ((uint32_t)sc >> 1) & 1u, abortp, p.status, 37)) { alive = false; break; }
-                tc_fence_after();
-                const uint32_t taddr = tmem_d + acc * 64 + ((uint32_t)(qq * 32) << 16);
-                __half* dst = dst0 + ((size_t)(y >> 1) * pl.W1s) * 128 + (y & 1) * 64;
+        Walk w;
+        w.start(p, g);
+        w.i = -1;                                         // forces the per-unit set-up at the first step
+        bool valid = false;
+        __half* dst0 = nullptr;
+        int unit_now = -1;
+        w.i = 0;
+        for (int k = g; k < total_steps; k += 2, w.pos += 2) {
+            w.settle(su);
+            if (w.i != unit_now) {
+                unit_now = w.i;
+                w.unit(p);
+                const int q = w.tile * kTileCols + 31 * qq + lane;
+                const int e = q / pl.Ws, X = q - e * pl.Ws;
+                valid = lane < 31 && e < p.n && X < pl.W1;
+                dst0 = p.out + ((size_t)e * pl.P1s + (X >> 1)) * 128 + (X & 1) * 32;
+            }
+            const int y = w.y_base + w.pos;
+            const int acc = k % NACC;
+            if (!mbar_wait_warp(&d_full[acc], ((uint32_t)(k / NACC)) & 1u, abortp, p.status, 37)) break;
+            tc_fence_after();
+            if (qq == 0 && lane == 0) {
+                // the MMAs of this step are complete: its two operand rows are free once the neighbouring step is
+                // done too (a row is read by two steps; the first and the last row of a unit by one, which
+                // then arrives for both)
+                const int r0 = k + w.i;
+                mbar_arrive(&a_empty[r0 % R]);
+                mbar_arrive(&a_empty[(r0 + 1) % R]);
+                if (w.pos == 0) mbar_arrive(&a_empty[r0 % R]);
+                if (w.pos == su - 1) mbar_arrive(&a_empty[(r0 + 1) % R]);
+            }
+            const uint32_t taddr = tmem_d + acc * 64 + ((uint32_t)(qq * 32) << 16);
+            uint32_t v0[32], v1[32];
+            tmem_ld_32x32(taddr, v0);                   // dx = 0 part of this column's output
+            tmem_ld_32x32(taddr + 32, v1);              // dx = 1 part of the output one column to the left
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&d_empty[acc]);
+            __half* dst = dst0 + ((size_t)(y >> 1) * pl.W1s) * 128 + (y & 1) * 64;
 #pragma unroll
-                for (int j = 0; j < 32; j += 16) {
-                    uint32_t v0[16], v1[16];
-                    tmem_ld_32x16(taddr + j, v0);               // dx = 0 part of this column's output
-                    tmem_ld_32x16(taddr + 32 + j, v1);          // dx = 1 part of the output one column to the left
-                    tmem_ld_wait();
-                    if (j == 16) {
-                        tc_fence_before();
-                        mbar_arrive(&d_empty[acc]);
-                    }
-                    uint32_t pk[8];
+            for (int j = 0; j < 32; j += 16) {
+                uint32_t pk[8];
 #pragma unroll
-                    for (int hh = 0; hh < 8; ++hh) {
-                        const int c = 2 * hh;
-                        const float a0 = __uint_as_float(v0[c]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c]), 1);
-                        const float a1 = __uint_as_float(v0[c + 1]) + __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c + 1]), 1);
-                        pk[hh] = relu_pack_h2(fmaf(a0, inv, s_bias[j + c]), fmaf(a1, inv, s_bias[j + c + 1]));
-                    }
-                    if (valid)
-                        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-                                     ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
-                                       "r"(pk[6]), "r"(pk[7]) : "memory");
+                for (int hh = 0; hh < 8; ++hh) {
+                    const int c = j + 2 * hh;
+                    float a0 = __uint_as_float(v0[c]), a1 = __uint_as_float(v0[c + 1]);
+                    add2(a0, a1, __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c]), 1),
+                         __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c + 1]), 1));
+                    fma2(a0, a1, inv, s_bias[c], s_bias[c + 1]);
+                    pk[hh] = relu_pack_h2(a0, a1);
                 }
+                if (valid)
+                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                   "r"(pk[6]), "r"(pk[7]) : "memory");
             }
         }
     }
@@ -302,7 +370,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const Conv1Params p)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_slot, (uint32_t)pl.tmem_cols);
+    if (warp == 1) tmem_dealloc(tmem_slot, 512);
 }
 
 __global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int C,
@@ -324,8 +392,9 @@ int choose_splits(int tiles, int H1, int grid)
     int best = 1;
     long best_cost = -1;
     for (int s = 1; s <= H1; ++s) {
-        const int steps = (H1 + s - 1) / s;
-        if (s > 1 && steps < 3) break;
+        if (H1 % s) continue;                              // equal ranges only
+        const int steps = H1 / s;
+        if (s > 1 && steps < 2) break;
         const long rounds = ((long)tiles * s + grid - 1) / grid;
         const long cost = rounds * (steps + 2);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
@@ -334,7 +403,8 @@ int choose_splits(int tiles, int H1, int grid)
 }
 
 template <int CG, int WC>
-hts_status launch_variant(const CUtensorMap& weight_map, const Conv1Params& p, int grid, int smem_bytes, cudaStream_t s)
+hts_status launch_variant(const CUtensorMap& weight_map, const CUtensorMap& frame_map, const Conv1Params& p, int grid,
+                          int smem_bytes, cudaStream_t s)
 {
     static int smem_set_by_device[kDeviceSlots] = {};
     int& smem_set = smem_set_by_device[device_slot()];
@@ -345,7 +415,7 @@ hts_status launch_variant(const CUtensorMap& weight_map, const Conv1Params& p, i
         HTS_CUDA(cudaFuncSetAttribute(conv1_march_kernel<CG, WC>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         smem_set = smem_bytes;
     }
-    HTS_CUDA(launch_pdl(conv1_march_kernel<CG, WC>, dim3(grid), dim3(kThreads), (size_t)smem_bytes, s, weight_map, p));
+    HTS_CUDA(launch_pdl(conv1_march_kernel<CG, WC>, dim3(grid), dim3(kThreads), (size_t)smem_bytes, s, weight_map, frame_map, p));
     note_launch();
     return HTS_OK;
 }
@@ -354,23 +424,24 @@ hts_status launch_variant(const CUtensorMap& weight_map, const Conv1Params& p, i
 
 bool conv1_plan(const Geometry& g, Conv1Plan* pl)
 {
-    // bulk copies of four input rows start and end on 16-byte boundaries when W is a multiple of 4
-    if (g.H % 4 || g.W % 4 || (g.C != 4 && g.C != 8 && g.C != 16)) return false;
+    // TMA boxes over the frames need 16-byte strides: H and W multiples of 4
+    if (g.H % 4 || g.W % 4 || (g.C != 4 && g.C != 8 && g.C != 16) || g.W > 1024) return false;
     pl->C = g.C; pl->H = g.H; pl->W = g.W; pl->CG = g.C / 4;
     pl->Hs = g.H / 4; pl->Ws = g.W / 4;
     pl->H1 = pl->Hs - 1; pl->W1 = pl->Ws - 1;
     if (pl->H1 != g.H1 || pl->W1 != g.W1 || pl->Ws < 2 || pl->H1 < 1) return false;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
     pl->env_max = kTileCols / pl->Ws + 2;
-    pl->stage_bytes = (pl->env_max * g.C * 4 * g.W + 127) / 128 * 128;
-    const bool two_per_sm = pl->CG == 1;
-    pl->ring = pl->CG == 4 ? 3 : 4;
-    pl->tmem_cols = two_per_sm ? 256 : 512;                    // 128 for the accumulators + ring x 32 CG
+    pl->group_rows = pl->CG == 1 ? 3 : 1;
+    pl->env_bytes = g.C * pl->group_rows * 4 * g.W;
+    pl->env_pitch = (pl->env_bytes + 127) / 128 * 128;
+    pl->stage_bytes = pl->env_max * pl->env_pitch;
+    pl->ring = pl->CG == 1 ? 8 : pl->CG == 2 ? 4 : 3;
+    pl->accs = pl->CG == 4 ? 2 : 4;                            // accs x 64 + ring x 32 CG <= 512 columns
     const int fixed = 1024 + 2 * pl->CG * kChunkBytes;
-    const int budget = (two_per_sm ? 112 : 226) * 1024 - fixed;
-    int st = budget / pl->stage_bytes;
+    int st = (226 * 1024 - fixed) / pl->stage_bytes;
     if (st > kMaxStages) st = kMaxStages;
-    if (st < 3) return false;
+    if (st < 2) return false;
     pl->stages = st;
     pl->smem_bytes = fixed + st * pl->stage_bytes;
     return true;
@@ -385,28 +456,43 @@ hts_status conv1_pack_weights(const Conv1Plan& pl, const __nv_bfloat16* w1, __ha
     return HTS_OK;
 }
 
-hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, const uint8_t* obs, const Indexing& ix, int n,
-                        const float* bias, const float* inv_scale, __half* out, int* status, cudaStream_t s)
+hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, Conv1MapCache& maps, const uint8_t* obs,
+                        const Indexing& ix, int n, const float* bias, const float* inv_scale, __half* out, int* status,
+                        cudaStream_t s)
 {
     const int sm_count = device_sm_count(device_slot());
     const long cols = (long)n * pl.Ws;
     if (cols >= (1L << 31) - 256) return HTS_ERR_INVALID_ARG;
+    // the tensor map over this frame buffer (dense: n frames; gathered: the whole pool)
+    const int frames = ix.slots ? ix.pool : n;
+    int slot = -1;
+    for (int i = 0; i < Conv1MapCache::kEntries; ++i)
+        if (maps.ptr[i] == obs && maps.frames[i] == frames) { slot = i; break; }
+    if (slot < 0) {
+        slot = maps.next;
+        maps.next = (maps.next + 1) % Conv1MapCache::kEntries;
+        if (!make_frames_map(&maps.map[slot], obs, pl.W, pl.H, pl.C, (uint64_t)frames, pl.group_rows)) {
+            maps.ptr[slot] = nullptr;
+            return HTS_ERR_CUDA;
+        }
+        maps.ptr[slot] = obs; maps.frames[slot] = frames;
+    }
     Conv1Params p{};
     p.pl = pl; p.obs = obs; p.slots = ix.slots; p.pool = ix.pool; p.n = n;
     p.tiles = (int)((cols + kTileCols - 1) / kTileCols);
-    const int per_sm = pl.CG == 1 ? 2 : 1;
-    const int max_grid = per_sm * sm_count;
-    p.splits = choose_splits(p.tiles, pl.H1, max_grid);
+    p.splits = choose_splits(p.tiles, pl.H1, sm_count);
+    p.su = pl.H1 / p.splits;
     p.bias = bias; p.inv_scale = inv_scale; p.out = out; p.status = status;
     const long units = (long)p.tiles * p.splits;
-    const int grid = units < max_grid ? (int)units : max_grid;
+    const int grid = units < sm_count ? (int)units : sm_count;
+    const CUtensorMap& fm = maps.map[slot];
     if (pl.CG == 1) {
-        if (pl.W == 84) return launch_variant<1, 84>(weight_map, p, grid, pl.smem_bytes, s);
-        return launch_variant<1, 0>(weight_map, p, grid, pl.smem_bytes, s);
+        if (pl.W == 84) return launch_variant<1, 84>(weight_map, fm, p, grid, pl.smem_bytes, s);
+        return launch_variant<1, 0>(weight_map, fm, p, grid, pl.smem_bytes, s);
     }
-    if (pl.CG == 2) return launch_variant<2, 0>(weight_map, p, grid, pl.smem_bytes, s);
-    if (pl.W == 96) return launch_variant<4, 96>(weight_map, p, grid, pl.smem_bytes, s);
-    return launch_variant<4, 0>(weight_map, p, grid, pl.smem_bytes, s);
+    if (pl.CG == 2) return launch_variant<2, 0>(weight_map, fm, p, grid, pl.smem_bytes, s);
+    if (pl.W == 96) return launch_variant<4, 96>(weight_map, fm, p, grid, pl.smem_bytes, s);
+    return launch_variant<4, 0>(weight_map, fm, p, grid, pl.smem_bytes, s);
 }
 
 }  // namespace hts

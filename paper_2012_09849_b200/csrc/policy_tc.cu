@@ -279,6 +279,7 @@ struct TcState {
     int splits, cps;            // FC split-K
     // packed weights
     Conv1Plan pl1;
+    Conv1MapCache maps1;
     __half *w1p, *w2p, *w3p, *wfcp;
     float *b1, *b2, *b3, *bfc, *whead, *bhead;
     unsigned* absmax;           // [L_COUNT]
@@ -364,7 +365,7 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
 {
     const Geometry& g = t->g;
     prof.begin(K_CONV1, s);
-    hts_status st = conv1_launch(t->pl1, t->mW1, obs, ix, n, t->b1, t->inv_scale + L_CONV1, t->a1s, t->status, s);
+    hts_status st = conv1_launch(t->pl1, t->mW1, t->maps1, obs, ix, n, t->b1, t->inv_scale + L_CONV1, t->a1s, t->status, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV1, s);
 

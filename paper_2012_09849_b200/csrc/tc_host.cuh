@@ -39,6 +39,20 @@ inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// uint8 frames [frames, C, H, W] seen as 32-bit words [frames][C][H/4 grid rows][W words]: the four input
+// rows under one grid row are W contiguous words.  Box = `group_rows` grid rows of all C channels of one frame.
+inline bool make_frames_map(CUtensorMap* m, const void* ptr, int W, int H, int C, uint64_t frames, int group_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)W, (cuuint64_t)(H / 4), (cuuint64_t)C, frames};
+    const cuuint64_t strides[3] = {(cuuint64_t)4 * W, (cuuint64_t)H * W, (cuuint64_t)C * H * W};
+    const cuuint32_t box[4] = {(cuuint32_t)W, (cuuint32_t)group_rows, (cuuint32_t)C, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 }  // namespace tc
 }  // namespace hts
