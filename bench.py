@@ -31,9 +31,10 @@ if ROOT not in sys.path:
 import hts_workloads as wl  # noqa: E402
 
 WORKLOAD = 3                       # hts_workloads.CONFIGS index
-# dram__bytes_read.sum + dram__bytes_write.sum of one conv1_ts_kernel<84> launch at this workload (n = 1024),
-# from the ncu capture summarised in profiles/actor_step_cfg3_n1024.md; reported only for that kernel
-CONV1_DRAM_TRAFFIC_BYTES = 28958720 + 126976
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of a kernel at this workload (n = 1024), from one ncu
+# capture of that kernel; None once the kernel has changed since its counters were taken
+DRAM_TRAFFIC_BYTES = {"conv1": None, "conv2": None, "conv3": None, "fc": None, "heads": None}
+DTYPE = "bf16 weights, fp16 operands, fp32 accumulate"
 METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
 UNIT = "env-steps/s"
 SEED = 0x5EED
@@ -230,6 +231,65 @@ def run_batch_sweep() -> None:
 
 
 # ------------------------------------------------------------------------------------------------
+def config_points(hts, torch, dev, peaks, stream, l2_bytes) -> dict:
+    """The other configurations on the same line: actor-step time at the configuration's own batch (frames from a
+    ring of device-generated batches larger than twice L2, same value law as the seeded recipe) and the advantage
+    scan at its own [T, N] with L2 flushed between launches."""
+    out = {}
+    flush = torch.empty(2 * l2_bytes, dtype=torch.uint8, device=dev)
+    for ci in (1, 2, 4):
+        c = wl.CONFIGS[ci]
+        n = c.N
+        dt = hts.HTS_DTYPE_FP32 if c.weight_dtype == "fp32" else hts.HTS_DTYPE_BF16
+        ctx = hts.hts_policy_create(c.C, c.H, c.W, c.A, dt, n)
+        hts.hts_policy_load_weights(ctx, hts.weights_to_device(wl.make_weights(c), dt, dev))
+        per_batch = n * c.C * c.H * c.W
+        ring = max(4, -(-2 * l2_bytes // per_batch))
+        g = torch.Generator(device=dev); g.manual_seed(1000 + ci)
+        if c.obs_law == "uniform":
+            frames = torch.randint(0, 256, (ring, n, c.C, c.H, c.W), dtype=torch.uint8, device=dev, generator=g)
+        else:
+            frames = ((torch.rand((ring, n, c.C, c.H, c.W), device=dev, generator=g) < 0.02) * 255).to(torch.uint8)
+        p_fr = [frames[i].data_ptr() for i in range(ring)]
+        ids = torch.arange(n, dtype=torch.int32, device=dev)
+        o = [torch.empty(n, dtype=torch.int32, device=dev)] + [torch.empty(n, device=dev) for _ in range(3)]
+        reps = 200 if n <= 256 else 100
+        for t in range(10):
+            hts.hts_policy_step(ctx, p_fr[t % ring], ids, None, t, SEED, n, *o, None, stream.cuda_stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for t in range(reps):
+            hts.hts_policy_step(ctx, p_fr[t % ring], ids, None, t, SEED, n, *o, None, stream.cuda_stream)
+        b.record(stream); torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(b) / reps
+        hts.hts_policy_destroy(ctx)
+        del frames
+        tf = 2.0 * macs_per_env_step(c) * n / (us * 1e-6) / 1e12
+        weight_bytes = (2 if dt == hts.HTS_DTYPE_BF16 else 4) * sum(int(np.prod(v.shape)) for v in wl.make_weights(c).values())
+        # the advantage scan at the configuration's own size, cold
+        r, v, d, bt = (torch.from_numpy(x).to(dev) for x in wl.make_rollout(c))
+        adv, ret = torch.empty_like(v), torch.empty_like(v)
+        g_ms = []
+        for i in range(12):
+            with torch.cuda.stream(stream):
+                flush.fill_(i)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            hts.hts_gae(r, v, d, bt, c.gamma, c.lam, c.T, c.N, adv, ret, stream)
+            b.record(stream); torch.cuda.synchronize()
+            g_ms.append(a.elapsed_time(b))
+        gae_us = 1e3 * float(np.median(g_ms[3:]))
+        out[f"cfg{ci}"] = {
+            "workload": c.name, "n": n, "obs": [c.C, c.H, c.W], "weights": c.weight_dtype, "ring_batches": ring,
+            "actor_step_us": us, "env_steps_per_s": n / (us * 1e-6), "tflops": tf,
+            "frac_of_bf16_burst": tf / peaks["bf16_tflops"], "frac_of_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+            "hbm_gbs_over_frames_and_weights": (per_batch + weight_bytes) / (us * 1e-6) / 1e9,
+            "gae": {"T": c.T, "N": c.N, "us_cold": gae_us, "elems_per_s": c.T * c.N / (gae_us * 1e-6),
+                    "gbs_cold": (17 * c.T * c.N + 4 * c.N) / (gae_us * 1e-6) / 1e9}}
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
 def run_ours(args) -> None:
     import torch
     import paper_2012_09849_b200 as hts
@@ -259,46 +319,18 @@ def run_ours(args) -> None:
     hts.hts_policy_load_weights(ctx, dev_w)
     obs_host = [torch.from_numpy(wl.make_obs(cfg, N, batch_index=i)).pin_memory() for i in range(ring)]
     obs_dev = [o.to(dev) for o in obs_host]
-    env_ids = torch.arange(rank * N, (rank + 1) * N, dtype=torch.int32, device=dev)
+    lo, hi = rank_env_range(rank, N)
+    env_ids = torch.arange(lo, hi, dtype=torch.int32, device=dev)
     r_np, _, d_np, _ = wl.make_rollout(cfg)
     rewards, dones = torch.from_numpy(r_np).to(dev), torch.from_numpy(d_np).to(dev)
 
-    class Storage:                                               # one of the two rollout storages
-        def __init__(self):
-            self.actions = torch.empty(T, N, dtype=torch.int32, device=dev)
-            self.logp = torch.empty(T, N, dtype=torch.float32, device=dev)
-            self.values = torch.empty(T, N, dtype=torch.float32, device=dev)
-            self.entropy = torch.empty(T, N, dtype=torch.float32, device=dev)
-            self.adv = torch.empty(T, N, dtype=torch.float32, device=dev)
-            self.ret = torch.empty(T, N, dtype=torch.float32, device=dev)
-            self.filled = torch.cuda.Event()                     # all T actor steps written
-            self.row0 = torch.cuda.Event()                       # value row 0 written
-            self.consumed = torch.cuda.Event()                   # GAE has read it
-            # raw row addresses, so the timed loop does no tensor slicing
-            self.p_act = [self.actions[t].data_ptr() for t in range(T)]
-            self.p_logp = [self.logp[t].data_ptr() for t in range(T)]
-            self.p_val = [self.values[t].data_ptr() for t in range(T)]
-            self.p_ent = [self.entropy[t].data_ptr() for t in range(T)]
-    store = [Storage(), Storage()]
-    s_act, s_gae = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    from paper_2012_09849_b200.pipeline import RolloutPipeline
     p_obs = [o.data_ptr() for o in obs_dev]
+    pipe = RolloutPipeline(ctx, T, N, env_ids, rewards, dones, cfg.gamma, cfg.lam,
+                           obs_for=lambda k, t: p_obs[(k * T + t) % ring], seed_for=lambda k: SEED + k, device=dev)
+    store, s_act, s_gae = pipe.store, pipe.s_act, pipe.s_gae
+    rollout = pipe.rollout
     p_ids, h_act_stream, h_gae_stream = env_ids.data_ptr(), s_act.cuda_stream, s_gae.cuda_stream
-
-    def rollout(k: int):
-        cur, prev = store[k % 2], store[(k + 1) % 2]
-        s_act.wait_event(cur.consumed)                           # storage free again (role swap)
-        for t in range(T):
-            hts.hts_policy_step(ctx, p_obs[(k * T + t) % ring], p_ids, None, t, SEED + k, N,
-                                cur.p_act[t], cur.p_logp[t], cur.p_val[t], cur.p_ent[t], None, h_act_stream)
-            if t == 0:
-                cur.row0.record(s_act)
-        cur.filled.record(s_act)
-        # GAE of the previous rollout on the second stream; bootstrap = V of this rollout's first states
-        s_gae.wait_event(prev.filled)
-        s_gae.wait_event(cur.row0)
-        hts.hts_gae(rewards, prev.values, dones, cur.p_val[0], cfg.gamma, cfg.lam, T, N, prev.adv, prev.ret,
-                    h_gae_stream)
-        prev.consumed.record(s_gae)
 
     def barrier():
         torch.cuda.synchronize()
@@ -306,8 +338,6 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for s in store:
-        s.consumed.record(s_gae); s.filled.record(s_act); s.row0.record(s_act)
     rollout(-1)                                                  # fills storage 1 so the first GAE has input
     for k in range(args.warmup):
         rollout(k)
@@ -319,9 +349,11 @@ def run_ours(args) -> None:
     launches0 = hts.hts_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(s_act)
+    host_t0 = time.perf_counter()
     for k in range(args.steps):
         rollout(args.warmup + k)
-    s_act.wait_stream(s_gae)
+    host_enqueue_us = 1e6 * (time.perf_counter() - host_t0) / (args.steps * T)    # host time to enqueue one actor step
+    pipe.join()
     e1.record(s_act)
     barrier()
     launches = hts.hts_launch_count() - launches0
@@ -416,20 +448,61 @@ def run_ours(args) -> None:
         upd_ms.append(a.elapsed_time(b))
     upd_wide_ms = float(np.median(upd_ms[3:]))
     upd_gbs = 22 * T * Nw / (upd_wide_ms * 1e-3) / 1e9
-    del rw, vw, dw, bw, aw, qw, hb
+    del hb
 
-    # ---- dominant kernel and its roofline
+    # ---- dominant kernel and its roofline (both the burst and the sustained measured peaks)
     macs = layer_macs(cfg)
     top = max(kern, key=lambda k: kern[k]["ms_total"])
     top_us = kern[top]["us_per_launch"]
     achieved_tf = 2.0 * macs[top] * N / (top_us * 1e-6) / 1e12
-    peak_tf = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved_tf / peak_tf, "peak_kind": peak_kind + " sustained",
-                "traffic": CONV1_DRAM_TRAFFIC_BYTES if top == "conv1" else None,
+    peak_tf, peak_burst = peaks["bf16_tflops_sustained"], peaks["bf16_tflops"]
+    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved_tf, "peak": peak_burst, "unit": "TFLOP/s",
+                "frac": achieved_tf / peak_burst, "frac_burst": achieved_tf / peak_burst,
+                "frac_sustained": achieved_tf / peak_tf, "peak_sustained": peak_tf,
+                "peak_kind": peak_kind + " burst (the timed region is a fraction of a second at full clocks)",
+                "traffic": DRAM_TRAFFIC_BYTES.get(top),
                 "algorithmic_bytes": N * obs_bytes if top == "conv1" else None,
                 "us_per_launch": top_us}
+    for name, kk in kern.items():
+        tf = 2.0 * macs[name] * N / (max(kk["us_per_launch"], 1e-9) * 1e-6) / 1e12
+        kk["tflops"] = tf
+        kk["frac_burst"] = tf / peak_burst
     whole_tf = 2.0 * macs_per_env_step(cfg) * value / world / 1e12
+
+    # ---- overlap of the two streams: one rollout of actor steps and the advantage scan of the widened storage
+    #      (long enough to matter), run one after the other on one stream and side by side on two
+    def timed(fn, reps=3):
+        ms = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(s_act)
+            fn()
+            b.record(s_act); torch.cuda.synchronize()
+            ms.append(a.elapsed_time(b))
+        return float(np.median(ms))
+
+    def actor_only():
+        for t in range(T):
+            hts.hts_policy_step(ctx, p_obs[t % ring], p_ids, None, t, SEED, N, store[0].p_act[t], store[0].p_logp[t],
+                                store[0].p_val[t], store[0].p_ent[t], None, h_act_stream)
+
+    def gae_wide(stream_handle):
+        hts.hts_gae(rw, vw, dw, bw, cfg.gamma, cfg.lam, T, Nw, aw, qw, stream_handle)
+
+    def serial():
+        actor_only(); gae_wide(h_act_stream)
+
+    def overlapped():
+        s_gae.wait_stream(s_act)
+        gae_wide(h_gae_stream)
+        actor_only()
+        s_act.wait_stream(s_gae)
+
+    overlap = {"actor_ms": timed(actor_only), "gae_ms": timed(lambda: gae_wide(h_act_stream)),
+               "serial_ms": timed(serial), "overlapped_ms": timed(overlapped),
+               "what": f"{T} actor steps of {N} rows and one advantage scan over [{T},{Nw}]"}
+    del rw, vw, dw, bw, aw, qw
 
     # ---- the executor-facing form: frames gathered by slot from a state buffer (one ring entry), outputs
     #      scattered to the same slots of a storage row; slots = a random permutation of the pool
@@ -518,6 +591,8 @@ def run_ours(args) -> None:
         hts.hts_policy_destroy(ctx5)
         del obs5
 
+    other_configs = config_points(hts, torch, dev, peaks, s_act, l2) if rank == 0 else None
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -525,7 +600,7 @@ def run_ours(args) -> None:
 
     # ---- the oracle on this host's cores, bounded sample
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if not args.no_cpu_baseline:
         from oracle import hts_oracle as orc
         wt = orc.Weights(params)
         rows, nsteps = 1024, 8
@@ -545,14 +620,16 @@ def run_ours(args) -> None:
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "N": N, "T": T, "obs": [cfg.C, cfg.H, cfg.W], "actions": A,
-                   "envs_per_gpu": N, "l2": f"observation ring of {ring} batches ({ring * N * obs_bytes >> 20} MiB) exceeds L2 "
-                   f"({l2 >> 20} MiB); GAE-alone timing flushes L2 between launches",
-                   "kernel_times": "second pass over the same rollouts with CUDA events around each kernel"},
+        "dtype": DTYPE, "data": "synthetic",
+        "config": {"workload": cfg.name, "N": N, "T": T, "obs": [cfg.C, cfg.H, cfg.W], "actions": A},
+        "notes": {"envs_per_gpu": N, "l2": f"observation ring of {ring} batches ({ring * N * obs_bytes >> 20} MiB) exceeds L2 "
+                  f"({l2 >> 20} MiB); advantage-scan-alone timings flush L2 between launches",
+                  "kernel_times": "second pass over the same rollouts with CUDA events around each kernel"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline,
         "whole_step_tflops": whole_tf, "whole_step_frac_of_bf16_sustained": whole_tf / peak_tf,
+        "whole_step_frac_of_bf16_burst": whole_tf / peak_burst,
+        "host_enqueue_us_per_actor_step": host_enqueue_us, "overlap": overlap, "configs": other_configs,
         "kernels": kern,
         "gae": {"us_cold": gae_us, "elems_per_s": T * N / (gae_us * 1e-6), "gbs_cold": gae_bytes / (gae_us * 1e-6) / 1e9,
                 "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
@@ -574,6 +651,23 @@ def run_ours(args) -> None:
         dist.destroy_process_group()
 
 
+def rank_env_range(rank: int, envs_per_rank: int) -> tuple[int, int]:
+    """Global environment ids of a rank: every rank runs the same per-rank workload on its own id range."""
+    return rank * envs_per_rank, (rank + 1) * envs_per_rank
+
+
+def spawn_command(gpus: int, argv: list[str], port: int | None = None) -> list[str]:
+    port = port or int(os.environ.get("MASTER_PORT", "29541"))
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def spawn_ranks(gpus: int, argv: list[str]) -> int:
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")             # the rank count and the transport show up in the log
+    return subprocess.call(spawn_command(gpus, argv), env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -589,7 +683,16 @@ def main():
     ap.add_argument("--ncu-learner-case", action="store_true",
                     help="profiling driver: the HBM-bound kernels (advantage scan, sample means, update) on 2^25 "
                          "transitions, twice each, and exit")
+    ap.add_argument("--dry-run-ranks", action="store_true",
+                    help="start the ranks as for a real run, print each rank's environment-id range and exit (no GPU work)")
     args = ap.parse_args()
+    if args.dry_run_ranks:
+        if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+            sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+        rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+        lo, hi = rank_env_range(rank, wl.CONFIGS[WORKLOAD].N)
+        print(json.dumps({"rank": rank, "world": world, "env_lo": lo, "env_hi": hi}), flush=True)
+        return
     if args.batch_sweep:
         run_batch_sweep()
     elif args.ncu_learner_case:
@@ -599,6 +702,9 @@ def main():
     elif args.impl == "reference":
         run_reference(args)
     else:
+        if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+            # started without a launcher: start one rank per GPU ourselves (same command line, under torchrun)
+            sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
         run_ours(args)
 
 

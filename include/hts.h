@@ -78,7 +78,18 @@ typedef struct {
 
 /* Create a context for one network geometry on the current device.  Allocates the
  * packed-weight store and an activation workspace sized for max_batch (device
- * memory, freed by hts_policy_destroy).  Errors: INVALID_ARG, SHAPE, ALLOC, CUDA. */
+ * memory, freed by hts_policy_destroy).
+ * A HTS_DTYPE_BF16 context (tensor-core kernels) takes C in {4, 8, 16} and frames
+ * up to 260 pixels wide (the resident activation tiles of the second convolution
+ * must fit 227 KB of shared memory); anything else is refused here with
+ * HTS_ERR_SHAPE, before any device call, never at step time.  Its frame buffers (obs, state_buffer) must start on a
+ * 16-byte boundary (they are staged by TMA); a misaligned pointer is refused with
+ * HTS_ERR_INVALID_ARG by the step calls.  Activations between layers are fp16: a
+ * hidden activation above 65504 saturates there.  With |w| summed per output unit
+ * S1, S2, S3 for the three convolutions and biases b, the largest possible
+ * activation is bounded by S3 (S2 (S1 + |b1|) + |b2|) + |b3| (inputs lie in [0, 1]);
+ * He-initialised weights of this network stay near 2e4, see tests.
+ * Errors: INVALID_ARG, SHAPE, ALLOC, CUDA.                                         */
 hts_status hts_policy_create(const hts_net_desc *desc, hts_ctx **out);
 
 /* Repack the caller's weights into the library's internal layouts on `cuda_stream`.
@@ -257,10 +268,15 @@ hts_status hts_gae(const float *rewards, const float *values, const uint8_t *don
                    float *advantages, float *returns, void *cuda_stream);
 
 /* Same with HOST buffers; copies in, computes, copies out and waits.  Staging
- * memory is a library-owned device buffer that grows on demand (not thread safe). */
+ * memory is a library-owned device buffer per device that grows on demand (not
+ * thread safe) and stays allocated until hts_gae_host_release.                     */
 hts_status hts_gae_host(const float *rewards, const float *values, const uint8_t *dones,
                         const float *bootstrap, float gamma, float lambda, int32_t T,
                         int32_t N, float *advantages, float *returns, void *cuda_stream);
+
+/* Frees the staging buffer of hts_gae_host on the current device (waits for the
+ * device first).  The next hts_gae_host allocates again.  Errors: CUDA.           */
+hts_status hts_gae_host_release(void);
 
 /* The actor step for callers that must not allocate.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)

@@ -274,3 +274,37 @@ def ppo_terms(logp_new, logp_old, values, entropy, advantages, returns, clip: fl
         ent += h[i]
         frac += 1.0 if abs(rho - 1.0) > clip else 0.0
     return sur / n, vl / n, ent / n, frac / n
+
+
+def vtrace(log_rhos, rewards, values, dones, bootstrap, gamma: float, lam: float, rho_bar: float, c_bar: float):
+    """V-trace targets and truncated-importance-sampling policy-gradient advantages over a [T, N] storage: the
+    off-policy correction of the systems the paper compares its delayed gradient with (Section 2, IMPALA;
+    Appendix C, Table A1 "Truncated I.S."), taken from the cited paper's definition (Espeholt et al. 2018,
+    Section 4.1, Eq. 1 and its Remark 1 recursion, and the policy-gradient term of Section 4.2):
+
+        rho_t = min(rho_bar, pi/mu),   c_t = lam * min(c_bar, pi/mu),   pi/mu = exp(log_rhos_t)
+        delta_t = rho_t (r_t + g_t V_{t+1} - V_t),          g_t = gamma (1 - d_t),  V_T = bootstrap
+        vs_t - V_t = delta_t + g_t c_t (vs_{t+1} - V_{t+1}),   vs_T = bootstrap
+        pg_t = rho_t (r_t + g_t vs_{t+1} - V_t)
+
+    Plain backward loop in fp64; `dones` as in the advantage scan (a done cuts both the bootstrap and the trace).
+    Returns (vs, pg_advantages) rounded to fp32.  Python loop over T, numpy over N."""
+    lr, r, v, b = _f64(log_rhos), _f64(rewards), _f64(values), _f64(bootstrap)
+    d = np.asarray(dones) != 0
+    T, N = r.shape
+    ratio = np.exp(lr)
+    rho = np.minimum(float(rho_bar), ratio)
+    c = float(lam) * np.minimum(float(c_bar), ratio)
+    vs = np.empty((T, N), np.float64)
+    pg = np.empty((T, N), np.float64)
+    diff_next = np.zeros(N, np.float64)            # vs_{t+1} - V_{t+1}
+    v_next = b.copy()
+    vs_next = b.copy()
+    for t in range(T - 1, -1, -1):
+        g = float(gamma) * np.where(d[t], 0.0, 1.0)
+        delta = rho[t] * (r[t] + g * v_next - v[t])
+        diff = delta + g * c[t] * diff_next
+        vs[t] = v[t] + diff
+        pg[t] = rho[t] * (r[t] + g * vs_next - v[t])
+        diff_next, v_next, vs_next = diff, v[t], vs[t]
+    return vs.astype(np.float32), pg.astype(np.float32)

@@ -107,6 +107,7 @@ hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspac
 
 // ---- the tensor-core path (bf16 weights) -------------------------------------------------------
 struct TcState;
+hts_status tc_check_geometry(const Geometry& g);          // HTS_ERR_SHAPE if the tensor-core kernels cannot take it (no CUDA call)
 hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** out,
                      bool (*alloc)(void* ctx, void** p, size_t bytes), void* alloc_ctx);
 void tc_destroy(TcState* t);

@@ -180,7 +180,7 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
     static int smem_set_by_device[kDeviceSlots] = {};
     int& smem_set = smem_set_by_device[dev];
     constexpr int NST = CPT == 2 ? 4 : 6;        // activation tiles in the ring: two being multiplied, the rest in flight
-    const int smem = 1024 + TAPS * CPT * kChunkBytes + NST * CPT * p.tile_rows * 128;
+    const int smem = conv_res_smem_bytes(TAPS, CPT, p.tile_rows);
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;
     if (smem > smem_set) {
         HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

@@ -23,6 +23,14 @@ struct ConvResParams {
 // rows of the activation tile for a largest tap shift
 inline int conv_res_tile_rows(int max_shift) { return (128 + max_shift + 7) / 8 * 8; }
 
+// Shared memory the kernel needs for (taps, planes per tap) and a tile of `tile_rows` rows: resident filter plus the
+// ring of activation tiles.  A geometry fits if this stays within 227 KB.
+inline int conv_res_smem_bytes(int taps, int cpt, int tile_rows)
+{
+    const int nst = cpt == 2 ? 4 : 6;
+    return 1024 + taps * cpt * 64 * 128 + nst * cpt * tile_rows * 128;
+}
+
 // TAPS x CPT = filter taps x 64-channel planes per tap: (4,2) for conv2 on the space-to-depth
 // grid, (9,1) for conv3.  act_map: box [tile_rows x 64]; weight_map: box [64 x 64].
 template <int TAPS, int CPT>

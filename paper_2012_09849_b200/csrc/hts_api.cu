@@ -118,6 +118,10 @@ hts_status run_step(hts_ctx* ctx, const uint8_t* obs, const Indexing& ix, const 
 
 }  // namespace
 
+// staging buffer of hts_gae_host, one per device; grows on demand, freed by hts_gae_host_release
+static char* g_gae_stage[kDeviceSlots] = {};
+static size_t g_gae_stage_bytes[kDeviceSlots] = {};
+
 extern "C" {
 
 hts_status hts_policy_create(const hts_net_desc* d, hts_ctx** out)
@@ -137,6 +141,10 @@ hts_status hts_policy_create(const hts_net_desc* d, hts_ctx** out)
     if (g.H2 < 3 || g.W2 < 3) return HTS_ERR_SHAPE;
     g.H3 = conv_out(g.H2, 3, 1); g.W3 = conv_out(g.W2, 3, 1);
     g.F = 64 * g.H3 * g.W3;
+    if (d->weight_dtype == HTS_DTYPE_BF16) {                 // shape limits of the tensor-core kernels, before any CUDA call
+        const hts_status gs = tc_check_geometry(g);
+        if (gs != HTS_OK) return gs;
+    }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError(), "cudaGetDevice");
 
@@ -382,11 +390,9 @@ hts_status hts_gae_host(const float* rewards, const float* values, const uint8_t
 {
     hts_status st = check_gae_args(rewards, values, dones, bootstrap, gamma, lambda, T, N, advantages, returns);
     if (st != HTS_OK) return st;
-    static char* stage_by_device[kDeviceSlots] = {};
-    static size_t stage_bytes_by_device[kDeviceSlots] = {};
     const int dev = device_slot();
-    char*& stage = stage_by_device[dev];
-    size_t& stage_bytes = stage_bytes_by_device[dev];
+    char*& stage = g_gae_stage[dev];
+    size_t& stage_bytes = g_gae_stage_bytes[dev];
     const size_t tn = (size_t)T * N;
     const size_t tn4 = (tn * 4 + 255) / 256 * 256, tn1 = (tn + 255) / 256 * 256, n4 = ((size_t)N * 4 + 255) / 256 * 256;
     const size_t need = 4 * tn4 + tn1 + n4;
@@ -412,6 +418,17 @@ hts_status hts_gae_host(const float* rewards, const float* values, const uint8_t
     HTS_CUDA(cudaMemcpyAsync(advantages, d_a, tn * 4, cudaMemcpyDeviceToHost, s));
     HTS_CUDA(cudaMemcpyAsync(returns, d_q, tn * 4, cudaMemcpyDeviceToHost, s));
     HTS_CUDA(cudaStreamSynchronize(s));
+    return HTS_OK;
+}
+
+hts_status hts_gae_host_release(void)
+{
+    const int dev = device_slot();
+    if (g_gae_stage[dev]) {
+        HTS_CUDA(cudaDeviceSynchronize());
+        HTS_CUDA(cudaFree(g_gae_stage[dev]));
+        g_gae_stage[dev] = nullptr; g_gae_stage_bytes[dev] = 0;
+    }
     return HTS_OK;
 }
 

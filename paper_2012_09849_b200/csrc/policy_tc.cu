@@ -292,13 +292,24 @@ struct TcState {
     int* status;
 };
 
+hts_status tc_check_geometry(const Geometry& g)
+{
+    Conv1Plan pl;
+    if (!conv1_plan(g, &pl)) return HTS_ERR_SHAPE;
+    const int rows2 = conv_res_tile_rows(pl.W1s + 1), rows3 = conv_res_tile_rows(2 * g.W2 + 2);
+    if (rows2 > 256 || rows3 > 256) return HTS_ERR_SHAPE;                    // TMA box height
+    if (conv_res_smem_bytes(4, 2, rows2) > 227 * 1024 || conv_res_smem_bytes(9, 1, rows3) > 227 * 1024) return HTS_ERR_SHAPE;
+    if (g.F % BK) return HTS_ERR_SHAPE;
+    return HTS_OK;
+}
+
 hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** out,
                      bool (*alloc)(void* ctx, void** p, size_t bytes), void* alloc_ctx)
 {
     TcState* t = new (std::nothrow) TcState();
     if (!t) return HTS_ERR_ALLOC;
     t->g = g; t->max_batch = max_batch; t->status = status;
-    if (!conv1_plan(g, &t->pl1)) { delete t; return HTS_ERR_SHAPE; }
+    if (tc_check_geometry(g) != HTS_OK || !conv1_plan(g, &t->pl1)) { delete t; return HTS_ERR_SHAPE; }
     t->H1s = t->pl1.H1s; t->W1s = t->pl1.W1s; t->P1s = t->pl1.P1s;
     t->P2 = g.H2 * g.W2; t->P3 = g.H3 * g.W3;
     const int chunks = g.F / BK;

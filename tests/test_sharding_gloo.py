@@ -62,3 +62,25 @@ def test_two_ranks_partition_actions_and_timing():
         assert p.exitcode == 0
     assert same, "actions changed with the partition"
     assert slow == 15.0
+
+
+def test_bench_starts_its_own_ranks_with_disjoint_env_ranges():
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself; each takes its own range of global
+    environment ids (checked with the dry-run switch, which stops before any GPU work)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    env["MASTER_PORT"] = str(port)
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--dry-run-ranks"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    rows = [json.loads(line) for line in out.stdout.splitlines() if line.startswith("{")]
+    assert sorted(r["rank"] for r in rows) == [0, 1] and all(r["world"] == 2 for r in rows)
+    n = wl.CONFIGS[3].N
+    spans = sorted((r["env_lo"], r["env_hi"]) for r in rows)
+    assert spans == [(0, n), (n, 2 * n)]
