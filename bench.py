@@ -349,10 +349,8 @@ def run_ours(args) -> None:
     launches0 = hts.hts_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(s_act)
-    host_t0 = time.perf_counter()
     for k in range(args.steps):
         rollout(args.warmup + k)
-    host_enqueue_us = 1e6 * (time.perf_counter() - host_t0) / (args.steps * T)    # host time to enqueue one actor step
     pipe.join()
     e1.record(s_act)
     barrier()
@@ -401,6 +399,19 @@ def run_ours(args) -> None:
         w_ms.append(a.elapsed_time(b))
     wide_ms = float(np.median(w_ms[3:]))
     wide_gbs = (17 * T * Nw + 4 * Nw) / (wide_ms * 1e-3) / 1e9
+    # the off-policy-corrected scan (V-trace / truncated importance sampling) on the same widened shape: 21 bytes per element
+    lw = torch.zeros_like(vw).uniform_(-0.5, 0.5)
+    pw = torch.empty_like(vw)
+    v_ms = []
+    for i in range(8):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s_gae)
+        hts.hts_vtrace(lw, rw, vw, dw, bw, cfg.gamma, cfg.lam, 1.0, 1.0, T, Nw, aw, pw, s_gae)
+        b.record(s_gae); torch.cuda.synchronize()
+        v_ms.append(a.elapsed_time(b))
+    vtrace_ms = float(np.median(v_ms[3:]))
+    vtrace_gbs = (21 * T * Nw + 4 * Nw) / (vtrace_ms * 1e-3) / 1e9
+    del lw, pw
     # the learner's sample means (policy term of Eq. 4, value loss, entropy) over the same widened storage
     # (16 bytes per transition) and over the configuration's own [T, N] storage
     out3 = torch.empty(3, dtype=torch.float32, device=dev)
@@ -498,6 +509,17 @@ def run_ours(args) -> None:
         gae_wide(h_gae_stream)
         actor_only()
         s_act.wait_stream(s_gae)
+
+    # host time to enqueue one actor step: a burst short enough not to fill the launch queue (a full queue makes
+    # the host wait for the GPU and the two times look alike), started on an idle device
+    torch.cuda.synchronize()
+    burst = 48
+    host_t0 = time.perf_counter()
+    for t in range(burst):
+        hts.hts_policy_step(ctx, p_obs[t % ring], p_ids, None, t, SEED, N, store[0].p_act[t], store[0].p_logp[t],
+                            store[0].p_val[t], store[0].p_ent[t], None, h_act_stream)
+    host_enqueue_us = 1e6 * (time.perf_counter() - host_t0) / burst
+    torch.cuda.synchronize()
 
     overlap = {"actor_ms": timed(actor_only), "gae_ms": timed(lambda: gae_wide(h_act_stream)),
                "serial_ms": timed(serial), "overlapped_ms": timed(overlapped),
@@ -634,6 +656,8 @@ def run_ours(args) -> None:
         "gae": {"us_cold": gae_us, "elems_per_s": T * N / (gae_us * 1e-6), "gbs_cold": gae_bytes / (gae_us * 1e-6) / 1e9,
                 "wide": {"T": T, "N": Nw, "ms": wide_ms, "gbs": wide_gbs, "elems_per_s": T * Nw / (wide_ms * 1e-3),
                          "frac_of_hbm": wide_gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}},
+        "vtrace": {"wide": {"T": T, "N": Nw, "ms": vtrace_ms, "gbs": vtrace_gbs, "elems_per_s": T * Nw / (vtrace_ms * 1e-3),
+                            "frac_of_hbm": vtrace_gbs / peaks["hbm_gbs"], "bytes_per_elem": 21}},
         "learner_terms": {"us_cold": terms_us, "elems": T * N,
                           "wide": {"elems": T * Nw, "ms": terms_wide_ms, "gbs": terms_wide_gbs,
                                    "frac_of_hbm": terms_wide_gbs / peaks["hbm_gbs"]},

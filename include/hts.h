@@ -267,6 +267,23 @@ hts_status hts_gae(const float *rewards, const float *values, const uint8_t *don
                    const float *bootstrap, float gamma, float lambda, int32_t T, int32_t N,
                    float *advantages, float *returns, void *cuda_stream);
 
+/* The off-policy-corrected form of the same scan: V-trace targets and the truncated-
+ * importance-sampling policy-gradient advantages (the corrections the paper compares
+ * its delayed gradient with: Section 2, IMPALA; Appendix C, Table A1 "Truncated I.S.";
+ * definition: Espeholt et al. 2018, Section 4.1 Eq. 1 and Section 4.2):
+ *   ratio_t = exp(log_rhos_t)   rho_t = min(rho_bar, ratio_t)   c_t = lambda min(c_bar, ratio_t)
+ *   delta_t = rho_t (r_t + g_t V_{t+1} - V_t)        g_t = gamma (1-d_t),  V_T = bootstrap
+ *   vs_t    = V_t + D_t,   D_t = delta_t + g_t c_t D_{t+1},   D_T = 0
+ *   pg_t    = rho_t (r_t + g_t vs_{t+1} - V_t),      vs_T = bootstrap
+ *   log_rhos DEVICE f32 [T,N]: log pi(a_t|s_t) - log mu(a_t|s_t) (learner minus behaviour);
+ *   rewards, values, dones, bootstrap as for hts_gae;  vs, pg_advantages DEVICE f32 [T,N] out.
+ * With log_rhos = 0 and rho_bar, c_bar >= 1 this is hts_gae: vs = returns, pg = advantages.
+ * 0 <= gamma, lambda <= 1; rho_bar, c_bar >= 0.  Errors: INVALID_ARG, CUDA.            */
+hts_status hts_vtrace(const float *log_rhos, const float *rewards, const float *values,
+                      const uint8_t *dones, const float *bootstrap, float gamma, float lambda,
+                      float rho_bar, float c_bar, int32_t T, int32_t N, float *vs,
+                      float *pg_advantages, void *cuda_stream);
+
 /* Same with HOST buffers; copies in, computes, copies out and waits.  Staging
  * memory is a library-owned device buffer per device that grows on demand (not
  * thread safe) and stays allocated until hts_gae_host_release.                     */

@@ -26,7 +26,7 @@ EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "h
            "hts_policy_evaluate", "hts_a2c_terms", "hts_ppo_terms", "hts_delayed_update",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
-           "hts_gae_host", "hts_gae_host_release", "hts_policy_step_noalloc", "hts_wait_selftest", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
+           "hts_gae_host", "hts_gae_host_release", "hts_vtrace", "hts_policy_step_noalloc", "hts_wait_selftest", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
 
 
 class HtsError(RuntimeError):
@@ -92,6 +92,8 @@ def lib():
         gae = [vp, vp, vp, vp, f32, f32, i32, i32, vp, vp, vp]
         L.hts_gae.argtypes = gae
         L.hts_gae_host.argtypes = gae
+        L.hts_vtrace.argtypes = [vp, vp, vp, vp, vp, f32, f32, f32, f32, i32, i32, vp, vp, vp]
+        L.hts_vtrace.restype = C.c_int
         L.hts_gae_host_release.argtypes = []
         L.hts_gae_host_release.restype = C.c_int
         L.hts_policy_step_noalloc.argtypes = [C.POINTER(hts_net_desc), C.POINTER(hts_weights)] + step[1:]
@@ -233,6 +235,13 @@ def hts_gae(rewards, values, dones, bootstrap, gamma, lam, T, N, advantages, ret
 def hts_gae_host(rewards, values, dones, bootstrap, gamma, lam, T, N, advantages, returns, stream=None) -> None:
     _check(lib().hts_gae_host(_ptr(rewards), _ptr(values), _ptr(dones), _ptr(bootstrap), float(gamma), float(lam),
                               int(T), int(N), _ptr(advantages), _ptr(returns), _stream(stream)), "hts_gae_host")
+
+
+def hts_vtrace(log_rhos, rewards, values, dones, bootstrap, gamma, lam, rho_bar, c_bar, T, N, vs, pg_advantages,
+               stream=None) -> None:
+    _check(lib().hts_vtrace(_ptr(log_rhos), _ptr(rewards), _ptr(values), _ptr(dones), _ptr(bootstrap), float(gamma),
+                            float(lam), float(rho_bar), float(c_bar), int(T), int(N), _ptr(vs), _ptr(pg_advantages),
+                            _stream(stream)), "hts_vtrace")
 
 
 def hts_gae_host_release() -> None:

@@ -141,4 +141,9 @@ hts_status launch_gae(const float* rewards, const float* values, const uint8_t* 
                       const float* bootstrap, float gamma, float lambda, int T, int N,
                       float* adv, float* ret, cudaStream_t s);
 
+// ---- V-trace / truncated importance sampling scan ---------------------------------------------
+hts_status launch_vtrace(const float* log_rhos, const float* rewards, const float* values, const uint8_t* dones,
+                         const float* bootstrap, float gamma, float lambda, float rho_bar, float c_bar, int T, int N,
+                         float* vs, float* pg, cudaStream_t s);
+
 }  // namespace hts

@@ -384,6 +384,21 @@ hts_status hts_gae(const float* rewards, const float* values, const uint8_t* don
                       static_cast<cudaStream_t>(cuda_stream));
 }
 
+hts_status hts_vtrace(const float* log_rhos, const float* rewards, const float* values, const uint8_t* dones,
+                      const float* bootstrap, float gamma, float lambda, float rho_bar, float c_bar, int32_t T, int32_t N,
+                      float* vs, float* pg_advantages, void* cuda_stream)
+{
+    hts_status st = check_gae_args(rewards, values, dones, bootstrap, gamma, lambda, T, N, vs, pg_advantages);
+    if (st != HTS_OK) return st;
+    if (!log_rhos || !(rho_bar >= 0.f) || !(c_bar >= 0.f)) return HTS_ERR_INVALID_ARG;      // NaN fails both
+    const size_t tn = (size_t)T * N;
+    const Range in[] = {{log_rhos, tn * 4}, {rewards, tn * 4}, {values, tn * 4}, {dones, tn}, {bootstrap, (size_t)N * 4}};
+    const Range outr[] = {{vs, tn * 4}, {pg_advantages, tn * 4}};
+    if (any_overlap(in, 5, outr, 2)) return HTS_ERR_INVALID_ARG;
+    return launch_vtrace(log_rhos, rewards, values, dones, bootstrap, gamma, lambda, rho_bar, c_bar, T, N, vs, pg_advantages,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
 hts_status hts_gae_host(const float* rewards, const float* values, const uint8_t* dones, const float* bootstrap,
                         float gamma, float lambda, int32_t T, int32_t N, float* advantages, float* returns,
                         void* cuda_stream)
