@@ -35,13 +35,29 @@ using namespace tc;
 
 namespace {
 
-#ifndef HTS_CONV1_ISSUERS
-#define HTS_CONV1_ISSUERS 4
-#endif
-constexpr int kIssuers = HTS_CONV1_ISSUERS;     // one thread issues an MMA every 60 clocks or so; a 128 x 64 x 16 one runs for 32
-constexpr int kConvWarp0 = kIssuers + 1;        // warp 0 stages, 1..kIssuers issue, then 8 converter and 8 epilogue warps
-constexpr int kEpiWarp0 = kConvWarp0 + 8;
-constexpr int kThreads = (kEpiWarp0 + 8) * 32;
+// Pipeline shape per channel-group count: NI issuing threads, CGR / EGR groups of four converter / epilogue
+// warps, NACC accumulators, R operand rows in the ring, KR grid rows per staged group.
+// The barriers carry one parity bit, so no role may get two phases ahead on any of them.  Each accumulator is
+// drained by one epilogue group in step order (EGR divides NACC).  It is filled by one issuing thread in step
+// order where NI divides NACC; with sixteen channels (NI = 4, NACC = 2) the ring keeps the order instead: step
+// k + 2 reads operand row k + 3, which takes the ring entry of row k and is written only after step k is done.
+template <int CG> struct Shape;
+template <> struct Shape<1> {
+    static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 4, R = 8, TMEM = 512, PER_SM = 1, KR = 3;
+};
+template <> struct Shape<2> {
+    static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 4, R = 4, TMEM = 512, PER_SM = 1, KR = 1;
+};
+template <> struct Shape<4> {       // 32 MMAs per step: tensor-bound
+    static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 2, R = 3, TMEM = 512, PER_SM = 1, KR = 1;
+};
+static_assert(Shape<1>::NACC % Shape<1>::NI == 0 && Shape<2>::NACC % Shape<2>::NI == 0, "one issuing thread per accumulator");
+static_assert(Shape<4>::NACC + 1 >= Shape<4>::R, "the ring must order steps that share an accumulator");
+static_assert(Shape<1>::NACC % Shape<1>::EGR == 0 && Shape<2>::NACC % Shape<2>::EGR == 0 && Shape<4>::NACC % Shape<4>::EGR == 0,
+              "one epilogue group per accumulator");
+template <int CG> __host__ __device__ constexpr int conv_warp0() { return 1 + Shape<CG>::NI; }          // warp 0 stages, then the issuers
+template <int CG> __host__ __device__ constexpr int epi_warp0() { return conv_warp0<CG>() + 4 * Shape<CG>::CGR; }
+template <int CG> __host__ __device__ constexpr int threads_of() { return (epi_warp0<CG>() + 4 * Shape<CG>::EGR) * 32; }
 constexpr int kTileCols = 124;                  // new grid columns per tile (4 quarters x 31; one more is shared)
 constexpr int kChunkBytes = 64 * 128;           // one filter K chunk: 64 rows (dx, o) x 64 fp16
 constexpr int kMaxStages = 8;
@@ -126,14 +142,17 @@ __device__ __forceinline__ void fma2(float& a0, float& a1, float m, float c0, fl
 // CG: groups of four channels.  WC: the frame width when known at compile time (the converter's loads then
 // use immediate offsets), 0 = any.
 template <int CG, int WC>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_of<CG>(), Shape<CG>::PER_SM)
 conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const Conv1Params p)
 {
     const Conv1Plan& pl = p.pl;
     constexpr int ACOLS = 32 * CG;                     // tensor-memory columns of one operand row
-    constexpr int KR = CG == 1 ? 3 : 1;                // grid rows per staged group (= pl.group_rows)
-    constexpr int NACC = CG == 4 ? 2 : 4;              // accumulators (= pl.accs)
-    constexpr int R = CG == 1 ? 8 : CG == 2 ? 4 : 3;   // operand rows in the ring (= pl.ring)
+    using S = Shape<CG>;
+    constexpr int KR = S::KR;                          // grid rows per staged group (= pl.group_rows)
+    constexpr int NACC = S::NACC;                      // accumulators (= pl.accs)
+    constexpr int R = S::R;                            // operand rows in the ring (= pl.ring)
+    constexpr int kIssuers = S::NI, kConvGroups = S::CGR, kEpiGroups = S::EGR;
+    constexpr int kConvWarp0 = conv_warp0<CG>(), kEpiWarp0 = epi_warp0<CG>(), kThreads = threads_of<CG>();
     const int W = WC ? WC : pl.W;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t w_bar, u8_full[kMaxStages], u8_empty[kMaxStages], a_full[kMaxRing], a_empty[kMaxRing],
@@ -153,7 +172,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
     if (threadIdx.x == 0) {
         mbar_init(&w_bar, 1);
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 8); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&u8_full[s], 1); mbar_init(&u8_empty[s], 4 * kConvGroups); }
         for (int s = 0; s < kMaxRing; ++s) { mbar_init(&a_full[s], 4); mbar_init(&a_empty[s], 2); }
         for (int s = 0; s < kMaxAcc; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 4); }
         abort_flag = 0;
@@ -162,7 +181,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         tma_prefetch_desc(&tmX);
     }
     if (threadIdx.x >= 32 && threadIdx.x < 64) s_bias[threadIdx.x - 32] = p.bias[threadIdx.x - 32];
-    if (warp == 1) tmem_alloc(&tmem_slot, 512);
+    if (warp == 1) tmem_alloc(&tmem_slot, S::TMEM);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -259,7 +278,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             int yr = 0;                                   // row inside the staged group
             for (int j = 0; j < ru; ++j, ++r) {
                 if (yr == 0 && !mbar_wait_warp(&u8_full[st], stph, abortp, p.status, 35)) { alive = false; break; }
-                if ((r & 1) == h) {
+                if (r % kConvGroups == h) {
                     const int s = r % R;
                     const uint8_t* src = s_u8 + st * pl.stage_bytes + off + yr * 4 * W;
 #pragma unroll
@@ -312,7 +331,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         __half* dst0 = nullptr;
         int unit_now = -1;
         w.i = 0;
-        for (int k = g; k < total_steps; k += 2, w.pos += 2) {
+        for (int k = g; k < total_steps; k += kEpiGroups, w.pos += kEpiGroups) {
             w.settle(su);
             if (w.i != unit_now) {
                 unit_now = w.i;
@@ -337,30 +356,61 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 if (w.pos == su - 1) mbar_arrive(&a_empty[(r0 + 1) % R]);
             }
             const uint32_t taddr = tmem_d + acc * 64 + ((uint32_t)(qq * 32) << 16);
-            uint32_t v0[32], v1[32];
-            tmem_ld_32x32(taddr, v0);                   // dx = 0 part of this column's output
-            tmem_ld_32x32(taddr + 32, v1);              // dx = 1 part of the output one column to the left
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&d_empty[acc]);
             __half* dst = dst0 + ((size_t)(y >> 1) * pl.W1s) * 128 + (y & 1) * 64;
+            if constexpr (kThreads * S::PER_SM <= 768) {
+                // registers allow it: the whole accumulator row in one round trip to tensor memory
+                uint32_t v0[32], v1[32];
+                tmem_ld_32x32(taddr, v0);                   // dx = 0 part of this column's output
+                tmem_ld_32x32(taddr + 32, v1);              // dx = 1 part of the output one column to the left
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&d_empty[acc]);
 #pragma unroll
-            for (int j = 0; j < 32; j += 16) {
-                uint32_t pk[8];
+                for (int j = 0; j < 32; j += 16) {
+                    uint32_t pk[8];
 #pragma unroll
-                for (int hh = 0; hh < 8; ++hh) {
-                    const int c = j + 2 * hh;
-                    float a0 = __uint_as_float(v0[c]), a1 = __uint_as_float(v0[c + 1]);
-                    add2(a0, a1, __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c]), 1),
-                         __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c + 1]), 1));
-                    fma2(a0, a1, inv, s_bias[c], s_bias[c + 1]);
-                    pk[hh] = relu_pack_h2(a0, a1);
+                    for (int hh = 0; hh < 8; ++hh) {
+                        const int c = j + 2 * hh;
+                        float a0 = __uint_as_float(v0[c]), a1 = __uint_as_float(v0[c + 1]);
+                        add2(a0, a1, __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c]), 1),
+                             __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c + 1]), 1));
+                        fma2(a0, a1, inv, s_bias[c], s_bias[c + 1]);
+                        pk[hh] = relu_pack_h2(a0, a1);
+                    }
+                    if (valid)
+                        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                     ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                       "r"(pk[6]), "r"(pk[7]) : "memory");
                 }
-                if (valid)
-                    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-                                 ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
-                                   "r"(pk[6]), "r"(pk[7]) : "memory");
+            } else {
+                // 64 registers per thread: sixteen output channels per round trip
+#pragma unroll
+                for (int j = 0; j < 32; j += 16) {
+                    uint32_t v0[16], v1[16];
+                    tmem_ld_32x16(taddr + j, v0);
+                    tmem_ld_32x16(taddr + 32 + j, v1);
+                    tmem_ld_wait();
+                    if (j == 16) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&d_empty[acc]);
+                    }
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int hh = 0; hh < 8; ++hh) {
+                        const int c = 2 * hh;
+                        float a0 = __uint_as_float(v0[c]), a1 = __uint_as_float(v0[c + 1]);
+                        add2(a0, a1, __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c]), 1),
+                             __shfl_down_sync(0xffffffffu, __uint_as_float(v1[c + 1]), 1));
+                        fma2(a0, a1, inv, s_bias[j + c], s_bias[j + c + 1]);
+                        pk[hh] = relu_pack_h2(a0, a1);
+                    }
+                    if (valid)
+                        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                     ::"l"(dst + j), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                                       "r"(pk[6]), "r"(pk[7]) : "memory");
+                }
             }
         }
     }
@@ -370,7 +420,7 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_slot, 512);
+    if (warp == 1) tmem_dealloc(tmem_slot, S::TMEM);
 }
 
 __global__ void pack_conv1_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int C,
@@ -415,7 +465,7 @@ hts_status launch_variant(const CUtensorMap& weight_map, const CUtensorMap& fram
         HTS_CUDA(cudaFuncSetAttribute(conv1_march_kernel<CG, WC>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
         smem_set = smem_bytes;
     }
-    HTS_CUDA(launch_pdl(conv1_march_kernel<CG, WC>, dim3(grid), dim3(kThreads), (size_t)smem_bytes, s, weight_map, frame_map, p));
+    HTS_CUDA(launch_pdl(conv1_march_kernel<CG, WC>, dim3(grid), dim3(threads_of<CG>()), (size_t)smem_bytes, s, weight_map, frame_map, p));
     note_launch();
     return HTS_OK;
 }
@@ -432,14 +482,15 @@ bool conv1_plan(const Geometry& g, Conv1Plan* pl)
     if (pl->H1 != g.H1 || pl->W1 != g.W1 || pl->Ws < 2 || pl->H1 < 1) return false;
     pl->H1s = (pl->H1 + 1) / 2; pl->W1s = (pl->W1 + 1) / 2; pl->P1s = pl->H1s * pl->W1s;
     pl->env_max = kTileCols / pl->Ws + 2;
-    pl->group_rows = pl->CG == 1 ? 3 : 1;
+    const bool twin = pl->CG == 1;                             // Shape<1>: two CTAs per SM
+    pl->group_rows = pl->CG == 1 ? Shape<1>::KR : pl->CG == 2 ? Shape<2>::KR : Shape<4>::KR;
     pl->env_bytes = g.C * pl->group_rows * 4 * g.W;
     pl->env_pitch = (pl->env_bytes + 127) / 128 * 128;
     pl->stage_bytes = pl->env_max * pl->env_pitch;
-    pl->ring = pl->CG == 1 ? 8 : pl->CG == 2 ? 4 : 3;
-    pl->accs = pl->CG == 4 ? 2 : 4;                            // accs x 64 + ring x 32 CG <= 512 columns
+    pl->ring = pl->CG == 1 ? Shape<1>::R : pl->CG == 2 ? Shape<2>::R : Shape<4>::R;
+    pl->accs = pl->CG == 1 ? Shape<1>::NACC : pl->CG == 2 ? Shape<2>::NACC : Shape<4>::NACC;   // accs x 64 + ring x 32 CG columns
     const int fixed = 1024 + 2 * pl->CG * kChunkBytes;
-    int st = (226 * 1024 - fixed) / pl->stage_bytes;
+    int st = ((twin ? 112 : 226) * 1024 - fixed) / pl->stage_bytes;
     if (st > kMaxStages) st = kMaxStages;
     if (st < 2) return false;
     pl->stages = st;
@@ -480,11 +531,12 @@ hts_status conv1_launch(const Conv1Plan& pl, const CUtensorMap& weight_map, Conv
     Conv1Params p{};
     p.pl = pl; p.obs = obs; p.slots = ix.slots; p.pool = ix.pool; p.n = n;
     p.tiles = (int)((cols + kTileCols - 1) / kTileCols);
-    p.splits = choose_splits(p.tiles, pl.H1, sm_count);
+    const int max_grid = (pl.CG == 1 ? Shape<1>::PER_SM : 1) * sm_count;
+    p.splits = choose_splits(p.tiles, pl.H1, max_grid);
     p.su = pl.H1 / p.splits;
     p.bias = bias; p.inv_scale = inv_scale; p.out = out; p.status = status;
     const long units = (long)p.tiles * p.splits;
-    const int grid = units < sm_count ? (int)units : sm_count;
+    const int grid = units < max_grid ? (int)units : max_grid;
     const CUtensorMap& fm = maps.map[slot];
     if (pl.CG == 1) {
         if (pl.W == 84) return launch_variant<1, 84>(weight_map, fm, p, grid, pl.smem_bytes, s);
