@@ -308,3 +308,91 @@ def vtrace(log_rhos, rewards, values, dones, bootstrap, gamma: float, lam: float
         pg[t] = rho[t] * (r[t] + g * vs_next - v[t])
         diff_next, v_next, vs_next = diff, v[t], vs[t]
     return vs.astype(np.float32), pg.astype(np.float32)
+
+
+def objective(wt: Weights, obs, actions, advantages, returns, value_coef: float, entropy_coef: float,
+              logp_old=None, clip: float = 0.0):
+    """The scalar the learner ascends (Section 3, Eq. 4 is its gradient estimator; Eq. 5 applies that gradient):
+
+        J-hat = (1/n) sum_i [ S_i - value_coef (R_i - V(s_i))^2 + entropy_coef H(pi(.|s_i)) ]
+
+    with S_i = log pi(a_i|s_i) A_i for the actor-critic update (advantages held fixed: they are data), or, with
+    `logp_old` and clip > 0, the clipped surrogate S_i = min(rho_i A_i, clip(rho_i, 1-clip, 1+clip) A_i),
+    rho_i = exp(log pi(a_i|s_i) - logp_old_i), of the PPO runs.  fp64, from the forward oracle."""
+    ev = evaluate_actions(wt, obs, actions)
+    adv, ret = _f64(advantages).ravel(), _f64(returns).ravel()
+    n = adv.size
+    if logp_old is None or clip <= 0:
+        s = ev["logp"] * adv
+    else:
+        rho = np.exp(ev["logp"] - _f64(logp_old).ravel())
+        s = np.minimum(rho * adv, np.clip(rho, 1.0 - clip, 1.0 + clip) * adv)
+    return float(np.sum(s - value_coef * (ret - ev["values"]) ** 2 + entropy_coef * ev["entropy"]) / n)
+
+
+def _conv_backward(x, w, dy, stride):
+    """Gradients of y[n,o,i,j] = b[o] + sum_{c,u,v} w[o,c,u,v] x[n,c,i s+u,j s+v] given dy: (dx, dw, db).
+    One term of the chain rule per filter tap, written with strided views."""
+    O, Cc, k, _ = w.shape
+    _, _, Ho, Wo = dy.shape
+    dx = np.zeros_like(x)
+    dw = np.empty_like(w)
+    for u in range(k):
+        for v in range(k):
+            xs = x[:, :, u:u + stride * Ho:stride, v:v + stride * Wo:stride]          # x[n,c,i s+u,j s+v]
+            dw[:, :, u, v] = np.einsum("noij,ncij->oc", dy, xs)
+            dx[:, :, u:u + stride * Ho:stride, v:v + stride * Wo:stride] += np.einsum("noij,oc->ncij", dy, w[:, :, u, v])
+    return dx, dw, dy.sum(axis=(0, 2, 3))
+
+
+def objective_grad(wt: Weights, obs, actions, advantages, returns, value_coef: float, entropy_coef: float,
+                   logp_old=None, clip: float = 0.0):
+    """Gradient of `objective` with respect to the twelve parameter tensors: the quantity Eq. 4 estimates and
+    Eq. 5 adds to the parameters.  Chain rule through the network of Appendix F.1 / F.2 in fp64, layer by layer:
+    heads (softmax and entropy derivatives in closed form), FC, the three convolutions; ReLU passes the gradient
+    where its output is positive.  -> dict name -> array shaped like the parameter."""
+    obs = np.ascontiguousarray(obs, dtype=np.uint8)
+    n = obs.shape[0]
+    f = policy_forward(wt, obs, taps=True)
+    a = np.asarray(actions, dtype=np.int64)
+    adv, ret = _f64(advantages).ravel(), _f64(returns).ravel()
+    W = wt.arr
+    logits, value = f["logits"], f["value"]
+    m = logits.max(axis=1, keepdims=True)
+    lse = m + np.log(np.exp(logits - m).sum(axis=1, keepdims=True))
+    logp = logits - lse                                   # [n, A]
+    p = np.exp(logp)
+    ent = -(p * logp).sum(axis=1)
+    onehot = np.zeros_like(p); onehot[np.arange(n), a] = 1.0
+    lpa = logp[np.arange(n), a]
+    # dS_i / dlogpi(a_i)
+    if logp_old is None or clip <= 0:
+        ds = adv.copy()
+    else:
+        rho = np.exp(lpa - _f64(logp_old).ravel())
+        unclipped_active = rho * adv <= np.clip(rho, 1.0 - clip, 1.0 + clip) * adv      # the min takes the first argument
+        ds = np.where(unclipped_active, rho * adv, 0.0)
+    # d logpi(a) / d logit_j = [j == a] - p_j ;  dH / d logit_j = -p_j (log p_j + H)
+    dlogits = (ds[:, None] * (onehot - p) - entropy_coef * p * (logp + ent[:, None])) / n
+    dvalue = 2.0 * value_coef * (ret - value) / n
+    g = {}
+    h = f["fc"]                                           # [n, 512], after ReLU
+    g["pi_w"] = dlogits.T @ h
+    g["pi_b"] = dlogits.sum(axis=0)
+    g["v_w"] = (dvalue[:, None] * h).sum(axis=0)[None, :]
+    g["v_b"] = np.array([dvalue.sum()])
+    dh = dlogits @ W["pi_w"] + dvalue[:, None] * W["v_w"]
+    dh = dh * (h > 0)
+    a3 = f["conv3"]
+    flat = a3.reshape(n, -1)                              # (c, h, w) order, as the FC weight's columns
+    g["fc_w"] = dh.T @ flat
+    g["fc_b"] = dh.sum(axis=0)
+    da3 = (dh @ W["fc_w"]).reshape(a3.shape) * (a3 > 0)
+    a2, a1 = f["conv2"], f["conv1"]
+    da2, g["conv3_w"], g["conv3_b"] = _conv_backward(a2, W["conv3_w"], da3, 1)
+    da2 = da2 * (a2 > 0)
+    da1, g["conv2_w"], g["conv2_b"] = _conv_backward(a1, W["conv2_w"], da2, 2)
+    da1 = da1 * (a1 > 0)
+    x = obs.astype(np.float64) / 255.0
+    _, g["conv1_w"], g["conv1_b"] = _conv_backward(x, W["conv1_w"], da1, 4)
+    return g

@@ -60,7 +60,9 @@ class RolloutPipeline:
         self.obs_for, self.seed_for, self.after_scan = obs_for, seed_for, after_scan
         self.store = [Storage(T, N, device), Storage(T, N, device)]
         self.s_act = torch.cuda.Stream(device)
-        self.s_gae = torch.cuda.Stream(device) if overlap else self.s_act
+        # the scan runs at high priority: its blocks take the SMs that the persistent actor kernels free at their
+        # tails instead of queueing behind the next actor kernel
+        self.s_gae = torch.cuda.Stream(device, priority=-1) if overlap else self.s_act
         for s in self.store:
             s.consumed.record(self.s_gae); s.filled.record(self.s_act); s.row0.record(self.s_act)
         self._p_ids = env_ids.data_ptr()
