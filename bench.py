@@ -615,6 +615,28 @@ def run_ours(args) -> None:
 
     other_configs = config_points(hts, torch, dev, peaks, s_act, l2) if rank == 0 else None
 
+    # ---- the learner's gradient (forward + backward on the fp32 path, CUDA cores, untuned) on one actor batch
+    grad_pt = None
+    if rank == 0:
+        ctxg = hts.hts_policy_create(cfg.C, cfg.H, cfg.W, A, hts.HTS_DTYPE_FP32, N)
+        hts.hts_policy_load_weights(ctxg, hts.weights_to_device(params, hts.HTS_DTYPE_FP32, dev))
+        grads = {k: torch.empty(v.shape, dtype=torch.float32, device=dev) for k, v in params.items()}
+        ga = torch.randint(0, A, (N,), dtype=torch.int32, device=dev)
+        gadv, gret = torch.randn(N, device=dev), torch.randn(N, device=dev)
+        g_ms = []
+        for i in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(s_act)
+            hts.hts_policy_gradient(ctxg, obs_dev[i % ring], ga, gadv, gret, None, 0.5, 0.01, 0.0, N, grads, s_act)
+            b.record(s_act); torch.cuda.synchronize()
+            g_ms.append(a.elapsed_time(b))
+        hts.hts_policy_destroy(ctxg)
+        gms = float(np.median(g_ms[1:]))
+        gflop = 3 * 2.0 * macs_per_env_step(cfg) * N / 1e9          # forward + data gradient + weight gradient
+        grad_pt = {"n": N, "ms": gms, "samples_per_s": N / (gms * 1e-3), "tflops_fp32": gflop / gms,
+                   "arithmetic": "fp32 CUDA cores, fixed-order sums", "flops_counted": "3 x forward"}
+        del grads
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -664,6 +686,7 @@ def run_ours(args) -> None:
                           "ppo_wide": {"elems": T * Nw, "ms": ppo_wide_ms, "gbs": ppo_wide_gbs,
                                        "frac_of_hbm": ppo_wide_gbs / peaks["hbm_gbs"],
                                        "bytes_per_elem": "24 (six arrays) + 2 x 4 (advantage mean and variance passes)"}},
+        "learner_gradient": grad_pt,
         "delayed_update": {"elems": T * Nw, "ms": upd_wide_ms, "gbs": upd_gbs, "frac_of_hbm": upd_gbs / peaks["hbm_gbs"]},
         "actor_step_us": 1e3 * ms / (args.steps * T),
         "indexed_actor_step_us": indexed_us,

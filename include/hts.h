@@ -158,6 +158,38 @@ hts_status hts_policy_evaluate(hts_ctx *ctx, const uint8_t *obs, const int32_t *
                                float *logp, float *values, float *entropy, float *logits_or_null,
                                void *cuda_stream);
 
+/* The twelve gradient tensors, shaped like hts_weights, all DEVICE f32 (written, not accumulated). */
+typedef struct {
+    float *conv1_w, *conv1_b;
+    float *conv2_w, *conv2_b;
+    float *conv3_w, *conv3_b;
+    float *fc_w, *fc_b;
+    float *pi_w, *pi_b;
+    float *v_w, *v_b;
+} hts_grads;
+
+/* The gradient the learner applies (Section 3: Eq. 4 is this gradient's estimator; Section 4.1, Eq. 5
+ * adds it to the parameters):  grads = d J-hat / d theta  at the context's current weights, with
+ *   J-hat = (1/n) sum_i [ S_i - value_coef (R_i - V(s_i))^2 + entropy_coef H(pi(.|s_i)) ]
+ *   S_i   = log pi(a_i|s_i) A_i                                  if logp_old is NULL or clip == 0
+ *           min(rho_i A_i, clip(rho_i, 1-clip, 1+clip) A_i),  rho_i = exp(log pi(a_i|s_i) - logp_old_i)  otherwise
+ * (the advantages are data: no gradient flows through them).  One forward pass over the n frames and one
+ * backward pass through the network of Appendix F.1 / F.2; ReLU passes the gradient where its output is
+ * positive.  Feed the result to hts_delayed_update (it is an ascent direction).
+ *   obs DEVICE u8 [n,C,H,W]; actions DEVICE i32 [n] in [0, num_actions); advantages, returns DEVICE f32 [n];
+ *   logp_old DEVICE f32 [n] or NULL; grads: twelve DEVICE f32 buffers, PyTorch layouts, overwritten.
+ * Only HTS_DTYPE_FP32 contexts (the learner's master weights are fp32; a bf16 actor context is refreshed
+ * from them through hts_delayed_update's bf16 output and hts_policy_load_weights): a bf16 context returns
+ * HTS_ERR_UNSUPPORTED.  fp32 CUDA-core arithmetic, every sum in a fixed order; written for a reproducible
+ * result, not tuned.  The first call on a context allocates the backward workspace (device memory, freed
+ * by hts_policy_destroy).  An action outside the range is not used as an index: that sample contributes
+ * nothing and hts_last_async_error reports INVALID_ARG.
+ * Errors: INVALID_ARG (NULL, n out of range, clip < 0, non-finite coefficient), UNSUPPORTED, ALLOC, CUDA.  */
+hts_status hts_policy_gradient(hts_ctx *ctx, const uint8_t *obs, const int32_t *actions,
+                               const float *advantages, const float *returns,
+                               const float *logp_old_or_null, float value_coef, float entropy_coef,
+                               float clip, int32_t n, const hts_grads *grads, void *cuda_stream);
+
 /* The three sample means the actor-critic update is built from (Section 3), over
  * `count` stored transitions in any layout (e.g. the whole [T,N] storage):
  *   out3[0] = (1/count) sum logp_i (returns_i - values_i)    policy term of Eq. 4 (its

@@ -23,7 +23,7 @@ STATUS_NAMES = ["HTS_OK", "HTS_ERR_INVALID_ARG", "HTS_ERR_SHAPE", "HTS_ERR_ALLOC
 WEIGHT_NAMES = ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "conv3_w", "conv3_b",
                 "fc_w", "fc_b", "pi_w", "pi_b", "v_w", "v_b")
 EXPORTS = ("hts_policy_create", "hts_policy_load_weights", "hts_policy_step", "hts_policy_step_indexed", "hts_policy_step_host",
-           "hts_policy_evaluate", "hts_a2c_terms", "hts_ppo_terms", "hts_delayed_update",
+           "hts_policy_evaluate", "hts_policy_gradient", "hts_a2c_terms", "hts_ppo_terms", "hts_delayed_update",
            "hts_policy_read_activation", "hts_action_uniforms", "hts_policy_profile", "hts_policy_profile_read",
            "hts_policy_kernel_name", "hts_last_async_error", "hts_policy_destroy", "hts_gae",
            "hts_gae_host", "hts_gae_host_release", "hts_vtrace", "hts_policy_step_noalloc", "hts_wait_selftest", "hts_launch_count", "hts_last_cuda_error", "hts_status_string")
@@ -43,6 +43,10 @@ class hts_net_desc(C.Structure):
 
 
 class hts_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class hts_grads(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
 
 
@@ -70,6 +74,8 @@ def lib():
         L.hts_policy_step_indexed.argtypes = [vp, vp, i32, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp, vp]
         L.hts_policy_evaluate.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.hts_policy_evaluate.restype = C.c_int
+        L.hts_policy_gradient.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, i32, C.POINTER(hts_grads), vp]
+        L.hts_policy_gradient.restype = C.c_int
         L.hts_a2c_terms.argtypes = [vp, vp, vp, vp, C.c_int64, vp, vp]
         L.hts_a2c_terms.restype = C.c_int
         L.hts_ppo_terms.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int64, f32, i32, vp, vp]
@@ -166,6 +172,15 @@ def hts_policy_step_indexed(ctx, state_buffer, pool, slots, env_ids, t_per_env, 
 def hts_policy_evaluate(ctx, obs, actions, n, logp, values, entropy, logits=None, stream=None) -> None:
     _check(lib().hts_policy_evaluate(ctx, _ptr(obs), _ptr(actions), int(n), _ptr(logp), _ptr(values), _ptr(entropy),
                                      _ptr(logits), _stream(stream)), "hts_policy_evaluate")
+
+
+def hts_policy_gradient(ctx, obs, actions, advantages, returns, logp_old, value_coef, entropy_coef, clip, n, grads: dict,
+                        stream=None) -> None:
+    """grads: name -> CUDA float32 tensor shaped like the parameter (overwritten)."""
+    g = hts_grads(**{k: _ptr(grads[k]) for k in WEIGHT_NAMES})
+    _check(lib().hts_policy_gradient(ctx, _ptr(obs), _ptr(actions), _ptr(advantages), _ptr(returns), _ptr(logp_old),
+                                     float(value_coef), float(entropy_coef), float(clip), int(n), C.byref(g),
+                                     _stream(stream)), "hts_policy_gradient")
 
 
 def hts_a2c_terms(logp, values, entropy, returns, count, out3, stream=None) -> None:

@@ -105,6 +105,14 @@ hts_status ref_convert_weights(const Geometry& g, int dtype, const hts_weights& 
 hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspace& ws,
                        const uint8_t* obs, const Indexing& ix, int* status, int n, Profiler& prof, cudaStream_t s);
 
+// ---- gradient of the learner objective on the fp32 path (backward.cu) ---------------------------
+constexpr int kBackwardChunks = 64;      // batch chunks whose partial weight gradients are added in index order
+size_t backward_workspace_floats(const Geometry& g, int max_batch);
+hts_status ref_backward(const Geometry& g, const RefWeights& w, const RefWorkspace& act, const uint8_t* obs, float* ws,
+                        const float* logits, const float* values, const int32_t* actions, const float* adv,
+                        const float* ret, const float* logp_old, float value_coef, float entropy_coef, float clip,
+                        int n, int max_batch, int* status, const hts_grads& out, cudaStream_t s);
+
 // ---- the tensor-core path (bf16 weights) -------------------------------------------------------
 struct TcState;
 hts_status tc_check_geometry(const Geometry& g);          // HTS_ERR_SHAPE if the tensor-core kernels cannot take it (no CUDA call)

@@ -35,9 +35,11 @@ struct hts_ctx {
     uint8_t* s_obs = nullptr;
     int32_t *s_ids = nullptr, *s_t = nullptr, *s_act = nullptr;
     float *s_logp = nullptr, *s_val = nullptr, *s_ent = nullptr, *s_logits = nullptr;
+    float* bw_ws = nullptr;       // backward workspace (allocated by the first hts_policy_gradient)
+    float *bw_logits = nullptr, *bw_logp = nullptr, *bw_val = nullptr, *bw_ent = nullptr;
     int* status = nullptr;        // device status word
     Profiler prof;
-    void* allocs[96];
+    void* allocs[112];
     int nalloc = 0;
 };
 
@@ -47,7 +49,7 @@ template <typename T>
 bool dev_alloc(hts_ctx* c, T** p, size_t count)
 {
     void* q = nullptr;
-    if (c->nalloc >= 96) return false;
+    if (c->nalloc >= 112) return false;
     if (cudaMalloc(&q, count * sizeof(T) + 256) != cudaSuccess) { cudaGetLastError(); return false; }
     c->allocs[c->nalloc++] = q;
     *p = static_cast<T*>(q);
@@ -241,6 +243,32 @@ hts_status hts_policy_evaluate(hts_ctx* ctx, const uint8_t* obs, const int32_t* 
     if (any_overlap(in, 2, outr, 4)) return HTS_ERR_INVALID_ARG;
     return run_step(ctx, obs, Indexing{}, nullptr, nullptr, 0, 0, n, nullptr, logp, values, entropy, logits_or_null,
                     static_cast<cudaStream_t>(cuda_stream), actions);
+}
+
+hts_status hts_policy_gradient(hts_ctx* ctx, const uint8_t* obs, const int32_t* actions, const float* advantages,
+                               const float* returns, const float* logp_old_or_null, float value_coef, float entropy_coef,
+                               float clip, int32_t n, const hts_grads* grads, void* cuda_stream)
+{
+    if (!ctx || !obs || !actions || !advantages || !returns || !grads) return HTS_ERR_INVALID_ARG;
+    float* const* gp = reinterpret_cast<float* const*>(grads);
+    for (int i = 0; i < 12; ++i) if (!gp[i]) return HTS_ERR_INVALID_ARG;
+    if (n < 1 || n > ctx->desc.max_batch) return HTS_ERR_INVALID_ARG;
+    if (!(clip >= 0.f) || !std::isfinite(clip) || !std::isfinite(value_coef) || !std::isfinite(entropy_coef)) return HTS_ERR_INVALID_ARG;
+    if (ctx->tc) return HTS_ERR_UNSUPPORTED;
+    if (!ctx->loaded) return HTS_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)ctx->desc.max_batch;
+    if (!ctx->bw_ws) {
+        bool ok = dev_alloc(ctx, &ctx->bw_ws, backward_workspace_floats(ctx->g, ctx->desc.max_batch));
+        ok = ok && dev_alloc(ctx, &ctx->bw_logits, nb * ctx->g.A) && dev_alloc(ctx, &ctx->bw_logp, nb);
+        ok = ok && dev_alloc(ctx, &ctx->bw_val, nb) && dev_alloc(ctx, &ctx->bw_ent, nb);
+        if (!ok) { ctx->bw_ws = nullptr; return HTS_ERR_ALLOC; }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    hts_status st = run_step(ctx, obs, Indexing{}, nullptr, nullptr, 0, 0, n, nullptr, ctx->bw_logp, ctx->bw_val, ctx->bw_ent,
+                             ctx->bw_logits, s, actions);
+    if (st != HTS_OK) return st;
+    return ref_backward(ctx->g, ctx->rw, ctx->rws, obs, ctx->bw_ws, ctx->bw_logits, ctx->bw_val, actions, advantages, returns,
+                        logp_old_or_null, value_coef, entropy_coef, clip, n, ctx->desc.max_batch, ctx->status, *grads, s);
 }
 
 hts_status hts_policy_step_host(hts_ctx* ctx, const uint8_t* obs, const int32_t* env_ids,
