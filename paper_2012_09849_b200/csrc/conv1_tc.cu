@@ -37,24 +37,26 @@ namespace {
 
 // Pipeline shape per channel-group count: NI issuing threads, CGR / EGR groups of four converter / epilogue
 // warps, NACC accumulators, R operand rows in the ring, KR grid rows per staged group.
-// The barriers carry one parity bit, so no role may get two phases ahead on any of them.  Each accumulator is
-// drained by one epilogue group in step order (EGR divides NACC).  It is filled by one issuing thread in step
-// order where NI divides NACC; with sixteen channels (NI = 4, NACC = 2) the ring keeps the order instead: step
-// k + 2 reads operand row k + 3, which takes the ring entry of row k and is written only after step k is done.
+// The barriers carry one parity bit, so every waiter must stay within one phase of the barrier it waits on:
+// NI + 1 <= R (see the issuing threads), EGR divides NACC (an accumulator is drained by one epilogue group, in step
+// order), and R <= NACC + 1 where issuing threads share an accumulator (NI does not divide NACC).
 template <int CG> struct Shape;
 template <> struct Shape<1> {
     static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 4, R = 8, TMEM = 512, PER_SM = 1, KR = 3;
 };
 template <> struct Shape<2> {
-    static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 4, R = 4, TMEM = 512, PER_SM = 1, KR = 1;
+    static constexpr int NI = 3, CGR = 2, EGR = 2, NACC = 4, R = 4, TMEM = 512, PER_SM = 1, KR = 1;
 };
 template <> struct Shape<4> {       // 32 MMAs per step: tensor-bound
-    static constexpr int NI = 4, CGR = 2, EGR = 2, NACC = 2, R = 3, TMEM = 512, PER_SM = 1, KR = 1;
+    static constexpr int NI = 2, CGR = 2, EGR = 2, NACC = 2, R = 3, TMEM = 512, PER_SM = 1, KR = 1;
 };
-static_assert(Shape<1>::NACC % Shape<1>::NI == 0 && Shape<2>::NACC % Shape<2>::NI == 0, "one issuing thread per accumulator");
-static_assert(Shape<4>::NACC + 1 >= Shape<4>::R, "the ring must order steps that share an accumulator");
-static_assert(Shape<1>::NACC % Shape<1>::EGR == 0 && Shape<2>::NACC % Shape<2>::EGR == 0 && Shape<4>::NACC % Shape<4>::EGR == 0,
-              "one epilogue group per accumulator");
+template <int CG> constexpr bool shape_ok()
+{
+    using S = Shape<CG>;
+    return S::NI + 1 <= S::R && S::NACC % S::EGR == 0 && (S::NACC % S::NI == 0 || S::R <= S::NACC + 1) &&
+           S::NACC * 64 + S::R * 32 * CG <= S::TMEM;
+}
+static_assert(shape_ok<1>() && shape_ok<2>() && shape_ok<4>(), "pipeline shape breaks the one-phase rule or the tensor-memory budget");
 template <int CG> __host__ __device__ constexpr int conv_warp0() { return 1 + Shape<CG>::NI; }          // warp 0 stages, then the issuers
 template <int CG> __host__ __device__ constexpr int epi_warp0() { return conv_warp0<CG>() + 4 * Shape<CG>::CGR; }
 template <int CG> __host__ __device__ constexpr int threads_of() { return (epi_warp0<CG>() + 4 * Shape<CG>::EGR) * 32; }
@@ -240,9 +242,15 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 const int r0 = k + w.i, r1 = r0 + 1;                       // operand rows of this step
                 const int s0 = r0 % R, s1 = r1 % R;
                 const int acc = k % NACC;
-                if (!mbar_wait(&d_empty[acc], (((uint32_t)(k / NACC)) & 1u) ^ 1u, abortp, p.status, 33)) break;
+                // Operands first, accumulator second.  A barrier carries one parity bit, so a waiting thread must be
+                // within one phase of it.  From one step of this thread to its next the operand rows advance by NI, or by
+                // NI + 1 across a unit boundary; with NI + 1 <= R the ring entries of this step last held rows that this
+                // thread's previous step or an earlier one has read, so their barriers are exactly one phase on.  Once
+                // the operands are there, all steps up to k + 1 - R are complete, so the step that last used this
+                // accumulator has been issued and the accumulator's barrier is at most one phase behind.
                 if (!mbar_wait(&a_full[s0], ((uint32_t)(r0 / R)) & 1u, abortp, p.status, 34)) break;
                 if (!mbar_wait(&a_full[s1], ((uint32_t)(r1 / R)) & 1u, abortp, p.status, 34)) break;
+                if (!mbar_wait(&d_empty[acc], (((uint32_t)(k / NACC)) & 1u) ^ 1u, abortp, p.status, 33)) break;
                 tc_fence_after();
                 const uint32_t d_addr = tmem_d + acc * 64;
 #pragma unroll
@@ -254,6 +262,12 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                         for (int kk = 0; kk < 4; ++kk)
                             mma_f16_ts(d_addr, a_addr + cg * 32 + 8 * kk, bdesc[dy][cg] + 2 * kk, idesc, (dy | cg | kk) != 0);
                 }
+                // an operand row is read by two steps (as the lower and as the upper grid row) and is free once both are
+                // done; the first and the last row of a unit are read by one step only, which then arrives for both
+                mma_commit(&a_empty[s0]);
+                mma_commit(&a_empty[s1]);
+                if (w.pos == 0) mma_commit(&a_empty[s0]);
+                if (w.pos == su - 1) mma_commit(&a_empty[s1]);
                 mma_commit(&d_full[acc]);
             }
         }
@@ -345,16 +359,6 @@ conv1_march_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             const int acc = k % NACC;
             if (!mbar_wait_warp(&d_full[acc], ((uint32_t)(k / NACC)) & 1u, abortp, p.status, 37)) break;
             tc_fence_after();
-            if (qq == 0 && lane == 0) {
-                // the MMAs of this step are complete: its two operand rows are free once the neighbouring step is
-                // done too (a row is read by two steps; the first and the last row of a unit by one, which
-                // then arrives for both)
-                const int r0 = k + w.i;
-                mbar_arrive(&a_empty[r0 % R]);
-                mbar_arrive(&a_empty[(r0 + 1) % R]);
-                if (w.pos == 0) mbar_arrive(&a_empty[r0 % R]);
-                if (w.pos == su - 1) mbar_arrive(&a_empty[(r0 + 1) % R]);
-            }
             const uint32_t taddr = tmem_d + acc * 64 + ((uint32_t)(qq * 32) << 16);
             __half* dst = dst0 + ((size_t)(y >> 1) * pl.W1s) * 128 + (y & 1) * 64;
             if constexpr (kThreads * S::PER_SM <= 768) {
