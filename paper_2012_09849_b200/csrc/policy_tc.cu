@@ -25,7 +25,6 @@
 #include "tc_host.cuh"
 #include "conv1_tc.cuh"
 #include "conv_res_tc.cuh"
-#include "conv_march_tc.cuh"
 
 namespace hts {
 using namespace tc;
@@ -221,25 +220,6 @@ __global__ void pack_conv3_kernel(const __nv_bfloat16* __restrict__ w, __half* _
     const int tap = k / 64, c = k % 64;
     wp[i] = scaled_h(w[(o * 64 + c) * 9 + tap], scale[L_CONV3]);
 }
-// conv2 for the march kernel: Wm[dy*128 + dx*64 + o][(uy*2+ux)*32 + c] = w2[o][c][2dy+uy][2dx+ux]
-__global__ void pack_conv2_march_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, const float* __restrict__ scale)
-{
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= 256 * 128) return;
-    const int row = i / 128, cp = i % 128;
-    const int dy = row >> 7, dx = (row >> 6) & 1, o = row & 63;
-    const int uy = (cp / 32) >> 1, ux = (cp / 32) & 1, c = cp % 32;
-    wp[i] = scaled_h(w[((o * 32 + c) * 4 + (2 * dy + uy)) * 4 + (2 * dx + ux)], scale[L_CONV2]);
-}
-// conv3 for the march kernel: Wm[dy*192 + dx*64 + o][c] = w3[o][c][dy][dx]
-__global__ void pack_conv3_march_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, const float* __restrict__ scale)
-{
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= 576 * 64) return;
-    const int row = i / 64, c = i % 64;
-    const int dy = row / 192, dx = (row % 192) / 64, o = row % 64;
-    wp[i] = scaled_h(w[(o * 64 + c) * 9 + dy * 3 + dx], scale[L_CONV3]);
-}
 // FC: Wp[o][pix*64 + c] = wfc[o][c*P3 + pix]   (activations are stored pixel-major, channel-minor)
 __global__ void pack_fc_kernel(const __nv_bfloat16* __restrict__ w, __half* __restrict__ wp, int P3, const float* __restrict__ scale)
 {
@@ -300,10 +280,6 @@ struct TcState {
     // packed weights
     Conv1Plan pl1;
     Conv1MapCache maps1;
-    bool march = false;         // conv2 / conv3 on the tensor-memory march kernels (else the flat-grid kernels)
-    ConvMarchPlan pl2m, pl3m;
-    __half *w2m = nullptr, *w3m = nullptr;
-    CUtensorMap mX2m, mW2m, mX3m, mW3m;
     __half *w1p, *w2p, *w3p, *wfcp;
     float *b1, *b2, *b3, *bfc, *whead, *bhead;
     unsigned* absmax;           // [L_COUNT]
@@ -359,17 +335,6 @@ hts_status tc_create(const Geometry& g, int max_batch, int* status, TcState** ou
          make_map(&t->mA3, t->a2, nb * t->P2, 64, 128, t->rows3) && make_map(&t->mB3, t->w3p, 64, 576, 1152, 64) &&
          make_map(&t->mAfc, t->a3, nb, g.F, (uint64_t)g.F * 2, BM) && make_map(&t->mBfc, t->wfcp, 512, g.F, (uint64_t)g.F * 2, 128);
     if (!ok) { delete t; return HTS_ERR_CUDA; }
-    // the march kernels for conv2 / conv3 where their plan fits (they always do for the paper's frames)
-    t->march = conv_march_plan(2, 2, 128, t->H1s, t->W1s, &t->pl2m) && conv_march_plan(3, 3, 64, g.H2, g.W2, &t->pl3m) &&
-               t->pl2m.Hout == g.H2 && t->pl2m.Wout == g.W2 && t->pl3m.Hout == g.H3 && t->pl3m.Wout == g.W3;
-    if (t->march) {
-        if (!(A(&t->w2m, (size_t)256 * 128) && A(&t->w3m, (size_t)576 * 64))) { delete t; return HTS_ERR_ALLOC; }
-        ok = make_pixels_map(&t->mX2m, t->a1s, 2, (uint64_t)t->P1s, nb, (uint32_t)t->W1s, (uint32_t)t->pl2m.env_max) &&
-             make_map(&t->mW2m, t->w2m, 256, 128, 256, 128) &&
-             make_pixels_map(&t->mX3m, t->a2, 1, (uint64_t)t->P2, nb, (uint32_t)g.W2, (uint32_t)t->pl3m.env_max) &&
-             make_map(&t->mW3m, t->w3m, 576, 64, 128, 192);
-        if (!ok) { delete t; return HTS_ERR_CUDA; }
-    }
     *out = t;
     return HTS_OK;
 }
@@ -395,10 +360,6 @@ hts_status tc_load_weights(TcState* t, const hts_weights& w, cudaStream_t s)
     if (st1 != HTS_OK) return st1;
     pack_conv2_kernel<<<nblk(64 * 512, 256), 256, 0, s>>>(bf(w.conv2_w), t->w2p, t->scale); HTS_LAUNCH_CHECK("pack_conv2");
     pack_conv3_kernel<<<nblk(64 * 576, 256), 256, 0, s>>>(bf(w.conv3_w), t->w3p, t->scale); HTS_LAUNCH_CHECK("pack_conv3");
-    if (t->march) {
-        pack_conv2_march_kernel<<<nblk(256 * 128, 256), 256, 0, s>>>(bf(w.conv2_w), t->w2m, t->scale); HTS_LAUNCH_CHECK("pack_conv2_march");
-        pack_conv3_march_kernel<<<nblk(576 * 64, 256), 256, 0, s>>>(bf(w.conv3_w), t->w3m, t->scale); HTS_LAUNCH_CHECK("pack_conv3_march");
-    }
     pack_fc_kernel<<<nblk((size_t)512 * g.F, 256), 256, 0, s>>>(bf(w.fc_w), t->wfcp, t->P3, t->scale); HTS_LAUNCH_CHECK("pack_fc");
     struct It { const void* p; float* q; size_t n; };
     const It items[] = {{w.conv1_b, t->b1, 32}, {w.conv2_b, t->b2, 64},
@@ -427,12 +388,7 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
     c.P_in = t->P1s; c.W_in = t->W1s; c.H_out = g.H2; c.W_out = g.W2; c.P_out = t->P2;
     c.bias = t->b2; c.out = t->a2; c.inv_scale = t->inv_scale + L_CONV2;
     prof.begin(K_CONV2, s);
-    if (t->march) {
-        const ConvMarchArgs a2{n, t->b2, t->inv_scale + L_CONV2, t->a2, t->status};
-        st = conv_march_launch(t->pl2m, t->mX2m, t->mW2m, a2, s);
-    } else {
-        st = conv_res_launch<4, 2>(t->mA2, t->mB2, c, s);
-    }
+    st = conv_res_launch<4, 2>(t->mA2, t->mB2, c, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV2, s);
     // conv3: 3x3 taps on [H2, W2] x 64 -> [H3, W3] x 64
@@ -441,12 +397,7 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
     c.P_in = t->P2; c.W_in = g.W2; c.H_out = g.H3; c.W_out = g.W3; c.P_out = t->P3;
     c.bias = t->b3; c.out = t->a3; c.inv_scale = t->inv_scale + L_CONV3;
     prof.begin(K_CONV3, s);
-    if (t->march) {
-        const ConvMarchArgs a3{n, t->b3, t->inv_scale + L_CONV3, t->a3, t->status};
-        st = conv_march_launch(t->pl3m, t->mX3m, t->mW3m, a3, s);
-    } else {
-        st = conv_res_launch<9, 1>(t->mA3, t->mB3, c, s);
-    }
+    st = conv_res_launch<9, 1>(t->mA3, t->mB3, c, s);
     if (st != HTS_OK) return st;
     prof.end(K_CONV3, s);
     GemmParams p{};

@@ -39,32 +39,6 @@ inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t co
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// fp16 activations [env][pixel][C] (C = 64 * chunks) as a tensor of rank 3 (chunks == 1) or 4: [64][chunks][pixels][envs].
-// Box = 64 channels x chunks x box_pixels x box_envs, 128-byte swizzle: every pixel chunk is one 128-byte row.
-inline bool make_pixels_map(CUtensorMap* m, const void* ptr, int chunks, uint64_t pixels, uint64_t envs, uint32_t box_pixels,
-                            uint32_t box_envs)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const uint64_t px_bytes = (uint64_t)chunks * 128;
-    if (chunks == 1) {
-        const cuuint64_t dims[3] = {64, pixels, envs};
-        const cuuint64_t strides[2] = {px_bytes, pixels * px_bytes};
-        const cuuint32_t box[3] = {64, box_pixels, box_envs};
-        const cuuint32_t estr[3] = {1, 1, 1};
-        return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-    }
-    const cuuint64_t dims[4] = {64, (cuuint64_t)chunks, pixels, envs};
-    const cuuint64_t strides[3] = {128, px_bytes, pixels * px_bytes};
-    const cuuint32_t box[4] = {64, (cuuint32_t)chunks, box_pixels, box_envs};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // uint8 frames [frames, C, H, W] seen as 32-bit words [frames][C][H/4 grid rows][W words]: the four input
 // rows under one grid row are W contiguous words.  Box = `group_rows` grid rows of all C channels of one frame.
 inline bool make_frames_map(CUtensorMap* m, const void* ptr, int W, int H, int C, uint64_t frames, int group_rows)
