@@ -174,6 +174,163 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem_d, TMEM_COLS);
 }
 
+
+// ---- FC for large batches: all K ranges of a tile in one CTA -----------------------------------------
+// The FC result is defined as  h = relu(bias + p_0 + p_1 + ... + p_{S-1}),  p_s = inv * (sum over the K chunks of
+// range s, accumulated in tensor memory in chunk order), the p_s added in index order in fp32.  Small batches
+// spread the S ranges over S CTAs (gemm_tc_kernel writes the p_s, the heads kernel adds them), which fills the
+// SMs.  Once there are enough 128 x 128 tiles to fill them anyway, one CTA runs the S ranges of its tile back to
+// back, alternating between two accumulators, and its epilogue warps keep the running sum in registers: the same
+// operations in the same order (explicitly rounded multiplies and adds, no fused forms), hence the same bits, but
+// the hidden layer leaves the chip once (2 KB per observation instead of S x 2 KB) and the copy pipeline never
+// drains between ranges.
+constexpr int FCL_STAGES = 6;
+constexpr int FCL_THREADS = 320;          // warp 0 copies, warp 1 issues, warps 2..9 epilogue (two per lane quarter, 64 columns each)
+
+struct FclParams {
+    int splits, cps;                      // K ranges and chunks per range
+    int n;                                // valid rows
+    const float* bias;                    // [512]
+    const float* inv_scale;
+    float* h;                             // [n][512]
+    int* status;
+};
+
+__global__ void __launch_bounds__(FCL_THREADS)
+fc_ranges_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FclParams p)
+{
+    constexpr int BN = 128;
+    constexpr int B_BYTES = BN * BK * 2;
+    constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[FCL_STAGES], empty_bar[FCL_STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ float s_bias[BN];
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    volatile int* abortp = &abort_flag;
+    const int total_chunks = p.splits * p.cps;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < FCL_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 8); }
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + BN) s_bias[threadIdx.x - 64] = p.bias[n0 + threadIdx.x - 64];
+    if (warp == 1) tmem_alloc(&tmem_base_slot, 2 * BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_slot;
+    pdl_wait();
+    pdl_trigger();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kc = 0; kc < total_chunks; ++kc) {
+                const int s = kc % FCL_STAGES;
+                const uint32_t ph = (uint32_t)(kc / FCL_STAGES) & 1u;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1u, abortp, p.status, 51)) break;
+                uint8_t* a_dst = tiles + s * STAGE_BYTES;
+                mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+                tma_load_2d(a_dst, &tmA, kc * BK, m0, &full_bar[s]);
+                tma_load_2d(a_dst + A_BYTES, &tmB, kc * BK, n0, &full_bar[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_f16(0, BM, BN);
+            int kc = 0;
+            bool alive = true;
+            for (int sp = 0; alive && sp < p.splits; ++sp) {
+                const int acc = sp & 1;
+                if (!mbar_wait(&acc_empty[acc], (((uint32_t)(sp >> 1)) & 1u) ^ 1u, abortp, p.status, 52)) break;
+                tc_fence_after();
+                for (int c = 0; c < p.cps; ++c, ++kc) {
+                    const int s = kc % FCL_STAGES;
+                    if (!mbar_wait(&full_bar[s], (uint32_t)(kc / FCL_STAGES) & 1u, abortp, p.status, 53)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = base + s * STAGE_BYTES;
+                    const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        mma_f16_ss(tmem_d + acc * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (c | k) != 0);
+                    mma_commit(&empty_bar[s]);
+                }
+                if (alive) mma_commit(&acc_full[acc]);
+            }
+        }
+    } else {
+        // epilogue warps 2..9: lane quarter warp % 4, columns [64 half, 64 half + 64) of the tile
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        const float inv = *p.inv_scale;
+        float sum[64];
+        bool ok = true;
+        for (int sp = 0; ok && sp < p.splits; ++sp) {
+            const int acc = sp & 1;
+            ok = mbar_wait_warp(&acc_full[acc], ((uint32_t)(sp >> 1)) & 1u, abortp, p.status, 54);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_d + acc * BN + half * 64 + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(taddr + c, v);
+                tmem_ld_wait();
+                if (c == 32) {                            // the accumulator is in registers: hand it back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[acc]);
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float t = __fmul_rn(__uint_as_float(v[j]), inv);           // p_s, as the split kernel stores it
+                    sum[c + j] = sp == 0 ? t : __fadd_rn(sum[c + j], t);              // added in index order, as the heads kernel does
+                }
+            }
+        }
+        if (ok) {
+            // bias, ReLU, and the block turned through shared memory (the pipeline stages are free by now) so that
+            // eight lanes write one full 128-byte line
+            float* stage = reinterpret_cast<float*>(tiles) + (warp - 2) * (32 * 36);
+            float* dst = p.h + (size_t)(m0 + q * 32) * 512 + n0 + half * 64;
+            const int rl = lane >> 3, c4 = (lane & 7) * 4;
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(stage + lane * 36 + j) =
+                        make_float4(fmaxf(__fadd_rn(sum[c + j], s_bias[half * 64 + c + j]), 0.f),
+                                    fmaxf(__fadd_rn(sum[c + j + 1], s_bias[half * 64 + c + j + 1]), 0.f),
+                                    fmaxf(__fadd_rn(sum[c + j + 2], s_bias[half * 64 + c + j + 2]), 0.f),
+                                    fmaxf(__fadd_rn(sum[c + j + 3], s_bias[half * 64 + c + j + 3]), 0.f));
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + rl;
+                    const float4 val = *reinterpret_cast<const float4*>(stage + rr * 36 + c4);
+                    if (m0 + q * 32 + rr < p.n) *reinterpret_cast<float4*>(dst + (size_t)rr * 512 + c + c4) = val;
+                }
+                __syncwarp();
+            }
+        }
+    }
+    if (*abortp) {                                      // give copies still in flight time to land
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_d, 2 * BN);
+}
+
 // ---- weight scaling and packing ---------------------------------------------------------------
 __global__ void absmax_kernel(const __nv_bfloat16* __restrict__ w, size_t n, unsigned* __restrict__ slot)
 {
@@ -277,6 +434,7 @@ struct TcState {
     int H1s, W1s, P1s;          // space-to-depth(2) grid of the conv1 output
     int P2, P3;
     int splits, cps;            // FC split-K
+    bool h_final = false;       // the last forward pass wrote the finished hidden layer (large-batch FC), not partials
     // packed weights
     Conv1Plan pl1;
     Conv1MapCache maps1;
@@ -406,8 +564,24 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
     p.taps = 1; p.cpt = g.F / BK; p.nk = t->cps; p.tap_shift[0] = 0;
     p.out_f32 = t->hpart; p.split_stride = (size_t)t->max_batch * 512; p.ldo = 512; p.inv_scale = t->inv_scale + L_FC;
     prof.begin(K_FC, s);
-    st = launch_gemm<128, EPI_SPLITK>(t->mAfc, t->mBfc, p, dim3(nblk(n, BM), 4, t->splits), s);
-    if (st != HTS_OK) return st;
+    // enough tiles to fill the SMs without splitting K across CTAs: run the K ranges of a tile in one CTA
+    t->h_final = (long)nblk(n, BM) * 4 >= device_sm_count(device_slot());
+    if (t->h_final) {
+        constexpr int smem = FCL_STAGES * (A_BYTES + 128 * BK * 2) + 1024;
+        static bool attr_set_by_device[kDeviceSlots] = {};
+        bool& attr_set = attr_set_by_device[device_slot()];
+        if (!attr_set) {
+            HTS_CUDA(cudaFuncSetAttribute(fc_ranges_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            HTS_CUDA(cudaFuncSetAttribute(fc_ranges_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+            attr_set = true;
+        }
+        const FclParams fp{t->splits, t->cps, n, t->bfc, t->inv_scale + L_FC, t->h, t->status};
+        HTS_CUDA(launch_pdl(fc_ranges_kernel, dim3(nblk(n, BM), 4), dim3(FCL_THREADS), (size_t)smem, s, t->mAfc, t->mBfc, fp));
+        note_launch();
+    } else {
+        st = launch_gemm<128, EPI_SPLITK>(t->mAfc, t->mBfc, p, dim3(nblk(n, BM), 4, t->splits), s);
+        if (st != HTS_OK) return st;
+    }
     prof.end(K_FC, s);
     return HTS_OK;
 }
@@ -416,6 +590,9 @@ hts_status tc_heads(TcState* t, const int32_t* env_ids, const int32_t* t_per_env
                     const Indexing& ix, int32_t* actions, float* logp, float* values, float* entropy, float* logits,
                     cudaStream_t s, const int32_t* given_actions)
 {
+    if (t->h_final)        // the FC kernel wrote relu(bias + sum of the K ranges) itself
+        return launch_heads(t->h, 1, 0, nullptr, t->whead, t->bhead, t->g.A, env_ids, t_per_env, tt, seed, n, ix, t->status,
+                            actions, logp, values, entropy, logits, nullptr, s, given_actions);
     return launch_heads(t->hpart, t->splits, (size_t)t->max_batch * 512, t->bfc, t->whead, t->bhead, t->g.A, env_ids,
                         t_per_env, tt, seed, n, ix, t->status, actions, logp, values, entropy, logits, t->h, s, given_actions);
 }
