@@ -564,8 +564,10 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
     p.taps = 1; p.cpt = g.F / BK; p.nk = t->cps; p.tap_shift[0] = 0;
     p.out_f32 = t->hpart; p.split_stride = (size_t)t->max_batch * 512; p.ldo = 512; p.inv_scale = t->inv_scale + L_FC;
     prof.begin(K_FC, s);
-    // enough tiles to fill the SMs without splitting K across CTAs: run the K ranges of a tile in one CTA
-    t->h_final = (long)nblk(n, BM) * 4 >= device_sm_count(device_slot());
+    // From 64 tiles on (n > 1920) one CTA per tile running all K ranges beats spreading the ranges over CTAs
+    // (measured: 89 against 91 us per step at n = 2048, 139 against 166 at n = 4096, 254 against 298 at n = 8192;
+    // at n = 1024 its 32 CTAs would each pull 1.6 MB through one SM's L2 port)
+    t->h_final = (long)nblk(n, BM) * 4 >= 64;
     if (t->h_final) {
         constexpr int smem = FCL_STAGES * (A_BYTES + 128 * BK * 2) + 1024;
         static bool attr_set_by_device[kDeviceSlots] = {};
