@@ -594,8 +594,18 @@ def run_ours(args) -> None:
         b5.record(s_act); torch.cuda.synchronize()
         us5 = 1e3 * a5.elapsed_time(b5) / reps
         tf5 = 2.0 * macs_per_env_step(c5) * nb / (us5 * 1e-6) / 1e12
+        hts.hts_policy_profile(ctx5, True)                       # per-kernel event times at this batch
+        for t in range(10):
+            hts.hts_policy_step(ctx5, obs5[t % 2], ids5, None, t, SEED, nb, *o5, None, h_act_stream)
+        torch.cuda.synchronize()
+        hts.hts_policy_profile(ctx5, False)
+        kern5 = {}
+        for i in range(5):
+            tot, cnt = hts.hts_policy_profile_read(ctx5, i)
+            kern5[hts.hts_policy_kernel_name(i)] = 1e3 * tot / max(cnt, 1)
         big = {"workload": c5.name, "n": nb, "us_per_step": us5, "env_steps_per_s": nb / (us5 * 1e-6), "tflops": tf5,
-               "frac_of_bf16_sustained": tf5 / peak_tf, "frac_of_bf16_burst": tf5 / peaks["bf16_tflops"]}
+               "frac_of_bf16_sustained": tf5 / peak_tf, "frac_of_bf16_burst": tf5 / peaks["bf16_tflops"],
+               "kernel_us": kern5}
         # the same pool served as the asynchronous executors would hand it over: a random permutation cut into
         # batches of random size 1..4096, each gathered from the state buffer and scattered into the storage row
         batches = [torch.from_numpy(b).to(dev) for b in wl.make_async_batches(c5, nb, 4096)]
