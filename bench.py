@@ -33,7 +33,7 @@ import hts_workloads as wl  # noqa: E402
 WORKLOAD = 3                       # hts_workloads.CONFIGS index
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of a kernel at this workload (n = 1024), from one ncu
 # capture of that kernel; None once the kernel has changed since its counters were taken
-DRAM_TRAFFIC_BYTES = {"conv1": None, "conv2": None, "conv3": None, "fc": None, "heads": None}
+DRAM_TRAFFIC_BYTES = {"conv1": 28953344 + 242432, "conv2": None, "conv3": None, "fc": None, "heads": None}
 DTYPE = "bf16 weights, fp16 operands, fp32 accumulate"
 METRIC = "actor env-steps/s (whole rollout: T actor steps + GAE)"
 UNIT = "env-steps/s"
