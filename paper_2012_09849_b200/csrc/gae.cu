@@ -31,9 +31,13 @@ template <int VEC> __device__ __forceinline__ typename VecT<VEC>::F pack(const f
 template <> __device__ __forceinline__ float pack<1>(const float* o) { return o[0]; }
 template <> __device__ __forceinline__ float4 pack<4>(const float* o) { return make_float4(o[0], o[1], o[2], o[3]); }
 
-// blockDim = (32, W).  Block b owns columns [b*32*VEC, (b+1)*32*VEC).  Time is walked from the
-// end in super-chunks of W*L rows; warp w owns rows [t0 + w*L, t0 + (w+1)*L) of the super-chunk.
-template <int VEC, int L>
+// blockDim = (32, W).  A warp is CY rows of 32/CY threads: thread (cx, cy) of warp w owns columns
+// [b*cols + cx*VEC, +VEC) (cols = 32/CY*VEC columns per block b) and chunk w*CY + cy of the super-chunk.  Time
+// is walked from the end in super-chunks of W*CY*L rows.  CY = 1 is a warp across 32*VEC columns; CY = 4 makes
+// blocks four times narrower (8 columns: still whole 32-byte sectors per row) so that a problem with few
+// columns spreads over four times as many SMs.  Chunk boundaries, and with them every rounding, do not depend
+// on CY or W.
+template <int VEC, int L, int CY>
 __global__ void __launch_bounds__(VEC == 4 ? 512 : 1024)
 gae_scan_kernel(const float* __restrict__ rewards, const float* __restrict__ values,
                 const uint8_t* __restrict__ dones, const float* __restrict__ bootstrap,
@@ -42,22 +46,23 @@ gae_scan_kernel(const float* __restrict__ rewards, const float* __restrict__ val
 {
     using F = typename VecT<VEC>::F;
     using B = typename VecT<VEC>::B;
-    extern __shared__ float smem[];                  // [W][32*VEC] S, then [W][32*VEC] P
-    const int W = blockDim.y;
-    const int w = threadIdx.y;
-    const int lane = threadIdx.x;
-    const int cols = 32 * VEC;
-    const long col = (long)blockIdx.x * cols + lane * VEC;
+    extern __shared__ float smem[];                  // [NC][cols] S, then [NC][cols] P
+    constexpr int CXW = 32 / CY;                     // threads of a warp along env
+    const int NC = blockDim.y * CY;                  // chunks of a super-chunk
+    const int cx = threadIdx.x % CXW;
+    const int w = threadIdx.y * CY + threadIdx.x / CXW;      // my chunk of the super-chunk
+    const int cols = CXW * VEC;
+    const long col = (long)blockIdx.x * cols + cx * VEC;
     const bool col_ok = col < N;                     // N % VEC == 0 is guaranteed by the launcher
     float* sS = smem;
-    float* sP = smem + W * cols;
+    float* sP = smem + NC * cols;
     const float gl = gamma * lambda;
 
     float carry_in[VEC];                             // advantage at the first row after this super-chunk
 #pragma unroll
     for (int k = 0; k < VEC; ++k) carry_in[k] = 0.f;
 
-    const int span = W * L;
+    const int span = NC * L;
     const int nsuper = (T + span - 1) / span;
     for (int sc = nsuper - 1; sc >= 0; --sc) {
         const int t_begin = sc * span + w * L;       // first row of my chunk
@@ -105,19 +110,19 @@ gae_scan_kernel(const float* __restrict__ rewards, const float* __restrict__ val
         __syncthreads();                             // previous super-chunk's readers are done
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
-            sS[w * cols + lane * VEC + k] = S[k];
-            sP[w * cols + lane * VEC + k] = P[k];
+            sS[w * cols + cx * VEC + k] = S[k];
+            sP[w * cols + cx * VEC + k] = P[k];
         }
         __syncthreads();
         // chain the chunk maps from the last chunk down; pick up my own incoming advantage
         float c[VEC], mine[VEC];
 #pragma unroll
         for (int k = 0; k < VEC; ++k) { c[k] = carry_in[k]; mine[k] = 0.f; }
-        for (int ww = W - 1; ww >= 0; --ww) {
+        for (int ww = NC - 1; ww >= 0; --ww) {
 #pragma unroll
             for (int k = 0; k < VEC; ++k) {
                 if (ww == w) mine[k] = c[k];
-                c[k] = sS[ww * cols + lane * VEC + k] + sP[ww * cols + lane * VEC + k] * c[k];
+                c[k] = sS[ww * cols + cx * VEC + k] + sP[ww * cols + cx * VEC + k] * c[k];
             }
         }
 #pragma unroll
@@ -145,20 +150,21 @@ gae_scan_kernel(const float* __restrict__ rewards, const float* __restrict__ val
     }
 }
 
-template <int VEC, int L>
+template <int VEC, int L, int CY>
 hts_status launch_t(const float* r, const float* v, const uint8_t* d, const float* b, float gamma,
                     float lambda, int T, int N, float* adv, float* ret, cudaStream_t s)
 {
     // Wide problems (VEC == 4) have all the parallelism they need across env: two chunks per block
     // measured best (86 % of the copy bandwidth at T=128, N=2^20).  Narrow ones cut time as finely
     // as a block allows.
-    int W = (T + L - 1) / L;
+    const int chunks = (T + L - 1) / L;
+    int W = (chunks + CY - 1) / CY;
     const int maxW = (VEC == 4) ? 2 : 32;
     if (W > maxW) W = maxW;
-    const int cols = 32 * VEC;
+    const int cols = 32 / CY * VEC;
     const unsigned blocks = (unsigned)((N + cols - 1) / cols);
-    const size_t smem = (size_t)2 * W * cols * sizeof(float);
-    gae_scan_kernel<VEC, L><<<blocks, dim3(32, W), smem, s>>>(r, v, d, b, gamma, lambda, T, N, adv, ret);
+    const size_t smem = (size_t)2 * W * CY * cols * sizeof(float);
+    gae_scan_kernel<VEC, L, CY><<<blocks, dim3(32, W), smem, s>>>(r, v, d, b, gamma, lambda, T, N, adv, ret);
     HTS_LAUNCH_CHECK("gae_scan_kernel");
     return HTS_OK;
 }
@@ -175,8 +181,11 @@ hts_status launch_gae(const float* rewards, const float* values, const uint8_t* 
     const bool vec4 = (N % 4 == 0) && aligned(rewards, 16) && aligned(values, 16) && aligned(dones, 4) &&
                       aligned(bootstrap, 16) && aligned(adv, 16) && aligned(ret, 16) &&
                       ((long)N * T >= (1L << 22));
-    if (vec4) return launch_t<4, 2>(rewards, values, dones, bootstrap, gamma, lambda, T, N, adv, ret, s);
-    return launch_t<1, 8>(rewards, values, dones, bootstrap, gamma, lambda, T, N, adv, ret, s);
+    if (vec4) return launch_t<4, 2, 1>(rewards, values, dones, bootstrap, gamma, lambda, T, N, adv, ret, s);
+    // few columns and many rows: 8-column blocks, four chunks per warp (same chunks, same bits, four times the SMs)
+    if ((N + 31) / 32 < device_sm_count(device_slot()) / 2 && T >= 4 * 8)
+        return launch_t<1, 8, 4>(rewards, values, dones, bootstrap, gamma, lambda, T, N, adv, ret, s);
+    return launch_t<1, 8, 1>(rewards, values, dones, bootstrap, gamma, lambda, T, N, adv, ret, s);
 }
 
 }  // namespace hts

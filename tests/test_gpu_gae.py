@@ -43,6 +43,22 @@ def test_wide_problems_take_the_vector_path(T, N):
     _check(r, v, d, b, 0.993, 0.95)
 
 
+@pytest.mark.parametrize("T,N", [(512, 512), (128, 1024), (300, 70), (37, 203), (1100, 24)])
+def test_narrow_blocks_give_the_bits_of_wide_ones(T, N):
+    # few columns take 8-column blocks; the same columns inside a wide scalar problem take 32-column blocks.
+    # Chunk boundaries are the same, so every output bit must be.
+    cfg = wl.CONFIGS[4]
+    r, v, d, b = wl.make_rollout(cfg, T=T, N=N, sub=77)
+    d = (np.random.default_rng(T * 7 + N).random((T, N)) < 0.02).astype(np.uint8)
+    adv, ret = _check(r, v, d, b, 0.993, 0.95)
+    reps = -(-4801 // N)                                 # wide enough for 32-column blocks, odd width: scalar columns
+    wide = [np.ascontiguousarray(np.tile(x, (1, reps))[:, :reps * N - 1]) for x in (r, v, d)]
+    bw = np.ascontiguousarray(np.tile(b, reps)[:reps * N - 1])
+    adv_w, ret_w = gpu_gae(wide[0], wide[1], wide[2], bw, 0.993, 0.95)
+    assert np.array_equal(adv_w[:, :N].view(np.int32), adv.view(np.int32))
+    assert np.array_equal(ret_w[:, :N].view(np.int32), ret.view(np.int32))
+
+
 def test_unaligned_wide_problem_falls_back():
     cfg = wl.CONFIGS[3]
     T, N = 64, 65537                                     # N % 4 != 0: scalar columns
