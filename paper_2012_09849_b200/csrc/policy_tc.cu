@@ -92,6 +92,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_slot;
+    // The weight halves of the first stages do not depend on the previous kernel: they are on their way while
+    // this one still waits for it.
+    if (warp == 0 && lane == 0) {
+        for (int kc = 0; kc < p.nk && kc < STAGES; ++kc) {
+            mbar_arrive_expect_tx(&full_bar[kc], STAGE_BYTES);
+            tma_load_2d(tiles + kc * STAGE_BYTES + A_BYTES, &tmB, (blockIdx.z * p.nk + kc) * BK, n0, &full_bar[kc]);
+        }
+    }
     pdl_wait();
     pdl_trigger();
 
@@ -104,9 +112,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int g = blockIdx.z * p.nk + kc;
                 const int tap = g / p.cpt, sub = g - tap * p.cpt;
                 uint8_t* a_dst = tiles + s * STAGE_BYTES;
-                mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+                if (kc >= STAGES) {
+                    mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+                    tma_load_2d(a_dst + A_BYTES, &tmB, g * BK, n0, &full_bar[s]);
+                }
                 tma_load_2d(a_dst, &tmA, sub * BK, m0 + p.tap_shift[tap], &full_bar[s]);
-                tma_load_2d(a_dst + A_BYTES, &tmB, g * BK, n0, &full_bar[s]);
             }
         }
     } else if (warp == 1) {
