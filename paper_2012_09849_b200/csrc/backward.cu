@@ -105,32 +105,49 @@ __global__ void dense_dgrad_kernel(const float* __restrict__ dout, int ldo, int 
 // Partial weight and bias gradients of a convolution over one chunk of the batch:
 //   part[chunk][p]  p < O C k k : sum_{i in chunk, y, x} dy[i][o][y][x] * in[i][c][y s + u][x s + v]
 //                   p >= O C k k: bias o = p - O C k k : sum dy[i][o][y][x]
+// A thread owns one (c, u, v) and kWgradOB output channels: one input load feeds that many independent
+// accumulators (the dy loads are the same address across most of a warp).  Each element is still summed over
+// (i, y, x) in ascending order.
+constexpr int kWgradOB = 8;
 template <typename TIn>
 __global__ void conv_wgrad_kernel(const float* __restrict__ dy, const TIn* __restrict__ in, int n, int C, int H, int W,
                                   int O, int k, int s, int Ho, int Wo, int per_chunk, float* __restrict__ part)
 {
-    const int nW = O * C * k * k, total = nW + O;
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= total) return;
+    const int per_o = C * k * k, nW = O * per_o, total = nW + O;
+    const int nT = nW / kWgradOB;                      // threads that own weights; O more own one bias each
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= nT + O) return;
     const int i0 = blockIdx.y * per_chunk;
     int i1 = i0 + per_chunk; i1 = i1 > n ? n : i1;
-    float acc = 0.f;
-    if (p < nW) {
-        const int v = p % k, u = (p / k) % k, c = (p / (k * k)) % C, o = p / (k * k * C);
+    float* out = part + (size_t)blockIdx.y * total;
+    const size_t plane = (size_t)Ho * Wo;
+    if (q < nT) {
+        const int r = q % per_o, o0 = (q / per_o) * kWgradOB;
+        const int v = r % k, u = (r / k) % k, c = r / (k * k);
+        float acc[kWgradOB];
+#pragma unroll
+        for (int j = 0; j < kWgradOB; ++j) acc[j] = 0.f;
         for (int i = i0; i < i1; ++i) {
-            const float* d = dy + ((size_t)i * O + o) * Ho * Wo;
+            const float* d = dy + ((size_t)i * O + o0) * plane;
             const TIn* x = in + ((size_t)i * C + c) * H * W + (size_t)u * W + v;
             for (int y = 0; y < Ho; ++y)
-                for (int xx = 0; xx < Wo; ++xx) acc = fmaf(d[y * Wo + xx], (float)x[(size_t)(y * s) * W + xx * s], acc);
+                for (int xx = 0; xx < Wo; ++xx) {
+                    const float xv = (float)x[(size_t)(y * s) * W + xx * s];
+#pragma unroll
+                    for (int j = 0; j < kWgradOB; ++j) acc[j] = fmaf(d[j * plane + y * Wo + xx], xv, acc[j]);
+                }
         }
+#pragma unroll
+        for (int j = 0; j < kWgradOB; ++j) out[(size_t)(o0 + j) * per_o + r] = acc[j];
     } else {
-        const int o = p - nW;
+        const int o = q - nT;
+        float acc = 0.f;
         for (int i = i0; i < i1; ++i) {
-            const float* d = dy + ((size_t)i * O + o) * Ho * Wo;
-            for (int q = 0; q < Ho * Wo; ++q) acc += d[q];
+            const float* d = dy + ((size_t)i * O + o) * plane;
+            for (int t = 0; t < Ho * Wo; ++t) acc += d[t];
         }
+        out[nW + o] = acc;
     }
-    part[(size_t)blockIdx.y * total + p] = acc;
 }
 
 // dW / db = in_scale * (chunk partials added in index order)
@@ -146,32 +163,59 @@ __global__ void conv_wgrad_reduce_kernel(const float* __restrict__ part, int chu
 }
 
 // dx[i][c][Y][X] = (x[i][c][Y][X] > 0) * sum_{o,u,v : Y = y s + u, X = x s + v} dy[i][o][y][x] * w[o][c][u][v]
-__global__ void conv_dgrad_kernel(const float* __restrict__ dy, const float* __restrict__ w, const float* __restrict__ x,
-                                  int n, int C, int H, int W, int O, int k, int s, int Ho, int Wo, float* __restrict__ dx)
+// A thread owns one input position and kDgradCB channels: every dy value it loads feeds that many independent
+// accumulators, and the block's slice of the filter sits in shared memory as [u][v][o][channel], so the inner loop
+// is one global load and two shared 16-byte loads per eight multiply-adds.  Taps are visited in ascending (u, v),
+// outputs in ascending o: the order of the sum of one element does not depend on the blocking.
+constexpr int kDgradCB = 8;
+__global__ void __launch_bounds__(256)
+conv_dgrad_kernel(const float* __restrict__ dy, const float* __restrict__ w, const float* __restrict__ x,
+                  int n, int C, int H, int W, int O, int k, int s, int Ho, int Wo, float* __restrict__ dx)
 {
-    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (size_t)n * C * H * W) return;
-    const int X = (int)(idx % W), Y = (int)((idx / W) % H), c = (int)((idx / ((size_t)W * H)) % C);
-    const size_t i = idx / ((size_t)W * H * C);
-    float acc = 0.f;
-    if (x[idx] > 0.f) {
-        for (int u = 0; u < k; ++u) {
-            const int yy = Y - u;
-            if (yy < 0 || yy % s) continue;
-            const int y = yy / s;
-            if (y >= Ho) continue;
-            for (int v = 0; v < k; ++v) {
-                const int xx = X - v;
-                if (xx < 0 || xx % s) continue;
-                const int xo = xx / s;
-                if (xo >= Wo) continue;
-                const float* d = dy + (i * O) * Ho * Wo + (size_t)y * Wo + xo;
-                const float* ww = w + ((size_t)c * k + u) * k + v;
-                for (int o = 0; o < O; ++o) acc = fmaf(d[(size_t)o * Ho * Wo], ww[(size_t)o * C * k * k], acc);
+    extern __shared__ float4 s_w4[];                   // [k*k][O][kDgradCB]
+    float* s_w = reinterpret_cast<float*>(s_w4);
+    const int c0 = blockIdx.y * kDgradCB;
+    for (int idx = threadIdx.x; idx < k * k * O * kDgradCB; idx += blockDim.x) {
+        const int cc = idx % kDgradCB, o = (idx / kDgradCB) % O, t = idx / (kDgradCB * O);
+        const int c = c0 + cc;
+        s_w[idx] = c < C ? w[((size_t)o * C + c) * k * k + t] : 0.f;
+    }
+    __syncthreads();
+    const size_t pos = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pos >= (size_t)n * H * W) return;
+    const int X = (int)(pos % W), Y = (int)((pos / W) % H);
+    const size_t i = pos / ((size_t)W * H);
+    float acc[kDgradCB];
+#pragma unroll
+    for (int cc = 0; cc < kDgradCB; ++cc) acc[cc] = 0.f;
+    const size_t plane = (size_t)Ho * Wo;
+    for (int u = Y % s; u < k && u <= Y; u += s) {
+        const int y = (Y - u) / s;
+        if (y >= Ho) continue;
+        for (int v = X % s; v < k && v <= X; v += s) {
+            const int xo = (X - v) / s;
+            if (xo >= Wo) continue;
+            const float* d = dy + i * O * plane + (size_t)y * Wo + xo;
+            const float4* wp = s_w4 + (size_t)(u * k + v) * O * (kDgradCB / 4);
+#pragma unroll 4
+            for (int o = 0; o < O; ++o) {
+                const float dv = d[(size_t)o * plane];
+                const float4 w0 = wp[2 * o], w1 = wp[2 * o + 1];
+                acc[0] = fmaf(dv, w0.x, acc[0]); acc[1] = fmaf(dv, w0.y, acc[1]);
+                acc[2] = fmaf(dv, w0.z, acc[2]); acc[3] = fmaf(dv, w0.w, acc[3]);
+                acc[4] = fmaf(dv, w1.x, acc[4]); acc[5] = fmaf(dv, w1.y, acc[5]);
+                acc[6] = fmaf(dv, w1.z, acc[6]); acc[7] = fmaf(dv, w1.w, acc[7]);
             }
         }
     }
-    dx[idx] = acc;
+#pragma unroll
+    for (int cc = 0; cc < kDgradCB; ++cc) {
+        const int c = c0 + cc;
+        if (c < C) {
+            const size_t idx = ((i * C + c) * H + Y) * W + X;
+            dx[idx] = x[idx] > 0.f ? acc[cc] : 0.f;
+        }
+    }
 }
 
 inline unsigned nblk(size_t total, int th) { return (unsigned)((total + th - 1) / th); }
@@ -232,18 +276,22 @@ hts_status ref_backward(const Geometry& g, const RefWeights& w, const RefWorkspa
         {da1, obs, true, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, w.w1, out.conv1_w, out.conv1_b, nullptr, nullptr}};
     for (const Layer& L : layers) {
         const int nW = L.O * L.C * L.k * L.k, total = nW + L.O;
+        if (L.O % kWgradOB) return HTS_ERR_SHAPE;
+        const int wthreads = nW / kWgradOB + L.O;
         if (L.u8)
-            conv_wgrad_kernel<uint8_t><<<dim3(nblk(total, 128), used), 128, 0, s>>>(
+            conv_wgrad_kernel<uint8_t><<<dim3(nblk(wthreads, 128), used), 128, 0, s>>>(
                 L.dy, static_cast<const uint8_t*>(L.in), n, L.C, L.H, L.W, L.O, L.k, L.s, L.Ho, L.Wo, per_chunk, part);
         else
-            conv_wgrad_kernel<float><<<dim3(nblk(total, 128), used), 128, 0, s>>>(
+            conv_wgrad_kernel<float><<<dim3(nblk(wthreads, 128), used), 128, 0, s>>>(
                 L.dy, static_cast<const float*>(L.in), n, L.C, L.H, L.W, L.O, L.k, L.s, L.Ho, L.Wo, per_chunk, part);
         HTS_LAUNCH_CHECK("conv_wgrad_kernel");
         conv_wgrad_reduce_kernel<<<nblk(total, th), th, 0, s>>>(part, used, nW, L.O, L.u8 ? 1.0f / 255.0f : 1.0f, L.dW, L.db);
         HTS_LAUNCH_CHECK("conv_wgrad_reduce_kernel");
         if (L.dx) {
-            conv_dgrad_kernel<<<nblk((size_t)n * L.C * L.H * L.W, th), th, 0, s>>>(L.dy, L.wt, L.x_act, n, L.C, L.H, L.W, L.O, L.k,
-                                                                                  L.s, L.Ho, L.Wo, L.dx);
+            const size_t w_smem = (size_t)L.k * L.k * L.O * kDgradCB * sizeof(float);
+            if (w_smem > 48 * 1024) return HTS_ERR_SHAPE;
+            conv_dgrad_kernel<<<dim3(nblk((size_t)n * L.H * L.W, 256), nblk(L.C, kDgradCB)), 256, w_smem, s>>>(
+                L.dy, L.wt, L.x_act, n, L.C, L.H, L.W, L.O, L.k, L.s, L.Ho, L.Wo, L.dx);
             HTS_LAUNCH_CHECK("conv_dgrad_kernel");
         }
     }
