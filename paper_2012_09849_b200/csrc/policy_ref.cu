@@ -1,6 +1,7 @@
 // fp32 CUDA-core path of the actor step: the check path (fp32 weights) of the policy-value
 // network of Appendix F.1 / F.2.  Direct convolution and dot products with fp32 FMAs and a
 // fixed summation order per output, so a row's result does not depend on the batch around it.
+#include <type_traits>
 #include "common.cuh"
 
 namespace hts {
@@ -15,19 +16,23 @@ __global__ void to_f32_kernel(const void* __restrict__ src, int dtype, float* __
 }
 
 // y[e,o,i,j] = relu(b[o] + sum_{c,u,v} w[o,c,u,v] * x[e,c,i*s+u,j*s+v]);  x is u8/255 or fp32.
-template <typename TIn>
+// A thread owns one output position and kConvOB output channels (O is a multiple of it): one input load feeds that
+// many accumulators, and the weight loads are one address per warp.  Every output is summed over (c, u, v) in
+// ascending order, whatever kConvOB: small batches take one channel per thread (more threads), large ones eight.
+template <typename TIn, int kConvOB>
 __global__ void conv_direct_kernel(const TIn* __restrict__ x, const float* __restrict__ w,
                                    const float* __restrict__ b, float* __restrict__ y,
                                    int n, int C, int H, int W, int O, int k, int s, int Ho, int Wo,
                                    float in_scale, const int32_t* __restrict__ slots, int pool, int* __restrict__ status)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const size_t total = (size_t)n * O * Ho * Wo;
+    const int OBn = O / kConvOB;
+    const size_t total = (size_t)n * OBn * Ho * Wo;
     if (idx >= total) return;
     const int j = (int)(idx % Wo);
     const int i = (int)((idx / Wo) % Ho);
-    const int o = (int)((idx / ((size_t)Wo * Ho)) % O);
-    const size_t e = idx / ((size_t)Wo * Ho * O);
+    const int o0 = (int)((idx / ((size_t)Wo * Ho)) % OBn) * kConvOB;
+    const size_t e = idx / ((size_t)Wo * Ho * OBn);
     size_t frame = e;                                   // dense, or the row's frame of the state buffer
     if (slots) {
         const int sl = slots[e];
@@ -35,16 +40,26 @@ __global__ void conv_direct_kernel(const TIn* __restrict__ x, const float* __res
         else frame = (size_t)sl;
     }
     const TIn* xe = x + frame * (size_t)C * H * W;
-    const float* wo = w + (size_t)o * C * k * k;
-    float acc = 0.f;
+    const size_t per_o = (size_t)C * k * k;
+    const float* wo = w + (size_t)o0 * per_o;
+    float acc[kConvOB];
+#pragma unroll
+    for (int q = 0; q < kConvOB; ++q) acc[q] = 0.f;
     for (int c = 0; c < C; ++c)
         for (int u = 0; u < k; ++u) {
             const TIn* xr = xe + ((size_t)c * H + (i * s + u)) * W + j * s;
             const float* wr = wo + (c * k + u) * k;
-            for (int v = 0; v < k; ++v) acc = fmaf(wr[v], (float)xr[v], acc);
+            for (int v = 0; v < k; ++v) {
+                const float xv = (float)xr[v];
+#pragma unroll
+                for (int q = 0; q < kConvOB; ++q) acc[q] = fmaf(wr[q * per_o + v], xv, acc[q]);
+            }
         }
-    acc = fmaf(acc, in_scale, b[o]);
-    y[idx] = acc > 0.f ? acc : 0.f;
+#pragma unroll
+    for (int q = 0; q < kConvOB; ++q) {
+        const float a = fmaf(acc[q], in_scale, b[o0 + q]);
+        y[((e * O + o0 + q) * Ho + i) * Wo + j] = a > 0.f ? a : 0.f;
+    }
 }
 
 // One warp per (env, output): h[e,o] = relu(b[o] + w[o,:] . x[e,:]); fixed lane-strided order.
@@ -92,19 +107,27 @@ hts_status ref_forward(const Geometry& g, const RefWeights& w, const RefWorkspac
                        const uint8_t* obs, const Indexing& ix, int* status, int n, Profiler& prof, cudaStream_t s)
 {
     const int th = 256;
+    auto conv = [&](auto* x, const float* wt, const float* b, float* y, int C, int H, int W, int O, int k, int st,
+                    int Ho, int Wo, float scale, const int32_t* slots, int pool, int* stat) {
+        using TIn = std::remove_cv_t<std::remove_pointer_t<decltype(x)>>;
+        const size_t outputs = (size_t)n * O * Ho * Wo;
+        if (outputs >= (size_t)8 * 2048 * 148)           // a thread for every eight outputs still fills the device
+            conv_direct_kernel<TIn, 8><<<blocks_for(outputs / 8, th), th, 0, s>>>(x, wt, b, y, n, C, H, W, O, k, st, Ho, Wo,
+                                                                               scale, slots, pool, stat);
+        else
+            conv_direct_kernel<TIn, 1><<<blocks_for(outputs, th), th, 0, s>>>(x, wt, b, y, n, C, H, W, O, k, st, Ho, Wo,
+                                                                            scale, slots, pool, stat);
+    };
     prof.begin(K_CONV1, s);
-    conv_direct_kernel<uint8_t><<<blocks_for((size_t)n * 32 * g.H1 * g.W1, th), th, 0, s>>>(
-        obs, w.w1, w.b1, ws.a1, n, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, 1.0f / 255.0f, ix.slots, ix.pool, status);
+    conv(obs, w.w1, w.b1, ws.a1, g.C, g.H, g.W, 32, 8, 4, g.H1, g.W1, 1.0f / 255.0f, ix.slots, ix.pool, status);
     HTS_LAUNCH_CHECK("conv1_direct");
     prof.end(K_CONV1, s);
     prof.begin(K_CONV2, s);
-    conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H2 * g.W2, th), th, 0, s>>>(
-        ws.a1, w.w2, w.b2, ws.a2, n, 32, g.H1, g.W1, 64, 4, 2, g.H2, g.W2, 1.0f, nullptr, 0, nullptr);
+    conv(static_cast<const float*>(ws.a1), w.w2, w.b2, ws.a2, 32, g.H1, g.W1, 64, 4, 2, g.H2, g.W2, 1.0f, nullptr, 0, nullptr);
     HTS_LAUNCH_CHECK("conv2_direct");
     prof.end(K_CONV2, s);
     prof.begin(K_CONV3, s);
-    conv_direct_kernel<float><<<blocks_for((size_t)n * 64 * g.H3 * g.W3, th), th, 0, s>>>(
-        ws.a2, w.w3, w.b3, ws.a3, n, 64, g.H2, g.W2, 64, 3, 1, g.H3, g.W3, 1.0f, nullptr, 0, nullptr);
+    conv(static_cast<const float*>(ws.a2), w.w3, w.b3, ws.a3, 64, g.H2, g.W2, 64, 3, 1, g.H3, g.W3, 1.0f, nullptr, 0, nullptr);
     HTS_LAUNCH_CHECK("conv3_direct");
     prof.end(K_CONV3, s);
     prof.begin(K_FC, s);
