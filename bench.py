@@ -150,13 +150,14 @@ def run_reference(args) -> None:
 
 
 # ------------------------------------------------------------------------------------------------
-def run_ncu_case(steps: int) -> None:
-    """A few actor steps of the bench workload (n = N rows each) and one GAE over [T, N]: the small case
-    that is captured under ncu.  Device footprint: two observation batches and the context (< 0.2 GB)."""
+def run_ncu_case(steps: int, rows: int = 0) -> None:
+    """A few actor steps of the bench workload (n = N rows each, or `rows` of the same frames and network) and
+    one GAE over [T, N]: the small case that is captured under ncu.  Device footprint: two observation batches
+    and the context (< 0.2 GB at 1024 rows, < 1 GB at 8192)."""
     import torch
     import paper_2012_09849_b200 as hts
     cfg = wl.CONFIGS[WORKLOAD]
-    T, N = cfg.T, cfg.N
+    T, N = cfg.T, (rows if rows > 0 else cfg.N)
     ctx = hts.hts_policy_create(cfg.C, cfg.H, cfg.W, cfg.A, hts.HTS_DTYPE_BF16, N)
     hts.hts_policy_load_weights(ctx, hts.weights_to_device(wl.make_weights(cfg), hts.HTS_DTYPE_BF16))
     obs = [torch.from_numpy(wl.make_obs(cfg, N, batch_index=i)).cuda() for i in range(2)]
@@ -165,7 +166,7 @@ def run_ncu_case(steps: int) -> None:
     f = [torch.empty(N, device="cuda") for _ in range(3)]
     for t in range(steps):
         hts.hts_policy_step(ctx, obs[t % 2], ids, None, t, SEED, N, act, *f)
-    r, v, d, b = (torch.from_numpy(x).cuda() for x in wl.make_rollout(cfg))
+    r, v, d, b = (torch.from_numpy(x).cuda() for x in wl.make_rollout(cfg, T=T, N=N))
     adv, ret = torch.empty_like(v), torch.empty_like(v)
     hts.hts_gae(r, v, d, b, cfg.gamma, cfg.lam, T, N, adv, ret)
     torch.cuda.synchronize()
@@ -735,6 +736,8 @@ def main():
     ap.add_argument("--ncu-case", type=int, default=0, metavar="STEPS",
                     help="profiling driver: run STEPS actor steps of the bench workload plus one GAE and exit "
                          "(no timing; for use under ncu)")
+    ap.add_argument("--ncu-rows", type=int, default=0, metavar="N",
+                    help="with --ncu-case: rows per actor step (default: the workload's N)")
     ap.add_argument("--batch-sweep", action="store_true",
                     help="print actor-step time against the batch size (1..8192) and exit")
     ap.add_argument("--ncu-learner-case", action="store_true",
@@ -755,7 +758,7 @@ def main():
     elif args.ncu_learner_case:
         run_ncu_learner_case()
     elif args.ncu_case > 0:
-        run_ncu_case(args.ncu_case)
+        run_ncu_case(args.ncu_case, args.ncu_rows)
     elif args.impl == "reference":
         run_reference(args)
     else:
