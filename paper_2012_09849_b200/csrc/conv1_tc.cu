@@ -99,14 +99,6 @@ __device__ __forceinline__ void u8x4_to_h4(uint32_t w, uint32_t& lo, uint32_t& h
     hi = __byte_perm(w, 0u, 0x4342);                    // {b2, 0, b3, 0}
 }
 
-// fp32 pair -> packed fp16 pair with ReLU, saturating at the largest finite fp16
-__device__ __forceinline__ uint32_t relu_pack_h2(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.relu.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
 // Position of a role in the CTA's sequence of units.  The CTA's units are u = blockIdx.x + i * gridDim.x; every
 // unit has `su` steps (output rows) and su + 1 grid rows, so a role that takes every k-th step or row of the
 // CTA's sequence finds its unit by stepping a counter instead of dividing.
@@ -128,18 +120,6 @@ struct Walk {
         return moved;
     }
 };
-
-// packed fp32 pairs (sm_100): two lanes of an add / fused multiply-add per instruction
-__device__ __forceinline__ void add2(float& a0, float& a1, float b0, float b1)
-{
-    asm("{\n\t.reg .b64 ra, rb;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
-        "add.rn.f32x2 ra, ra, rb;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
-}
-__device__ __forceinline__ void fma2(float& a0, float& a1, float m, float c0, float c1)
-{
-    asm("{\n\t.reg .b64 ra, rm, rc;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rm, {%2, %2};\n\tmov.b64 rc, {%3, %4};\n\t"
-        "fma.rn.f32x2 ra, ra, rm, rc;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(m), "f"(c0), "f"(c1));
-}
 
 // CG: groups of four channels.  WC: the frame width when known at compile time (the converter's loads then
 // use immediate offsets), 0 = any.

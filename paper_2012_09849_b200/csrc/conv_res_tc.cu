@@ -122,15 +122,23 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int r = q * 32 + lane;
         const float inv = *p.inv_scale;
         int it = grp;
+        // Row m of the flat grid = (env, y, x).  The row of this thread advances by the same amount from one of its
+        // tiles to the next, so (env, pix) are carried along with one conditional subtraction per tile instead of
+        // two divisions, and y = pix / W_in is a multiply: with pix < 2048 and W_in <= 64,
+        // (pix * ceil(2^20 / W_in)) >> 20 is exact and the product fits 32 bits (the launcher checks both bounds).
+        const uint32_t first = (uint32_t)(blockIdx.x + grp * gridDim.x) * 128u + (uint32_t)r;
+        const uint32_t stride = (uint32_t)kAcc * gridDim.x * 128u;
+        const int d_env = (int)(stride / (uint32_t)p.P_in), d_pix = (int)(stride - (uint32_t)d_env * (uint32_t)p.P_in);
+        int env = (int)(first / (uint32_t)p.P_in), pix = (int)(first - (uint32_t)env * (uint32_t)p.P_in);
+        const uint32_t w_magic = ((1u << 20) + (uint32_t)p.W_in - 1u) / (uint32_t)p.W_in;
         for (int tile = blockIdx.x + grp * gridDim.x; tile < tiles; tile += kAcc * gridDim.x, it += kAcc) {
             if (!mbar_wait_warp(&d_full[grp], ((uint32_t)(it / kAcc)) & 1u, abortp, p.status, 25)) break;
             tc_fence_after();
-            const uint32_t m = (uint32_t)tile * 128u + (uint32_t)r;       // < total_rows + 128, which fits 32 bits
-            const int env = (int)(m / (uint32_t)p.P_in);
-            const int pix = (int)(m - (uint32_t)env * (uint32_t)p.P_in);
-            const int y = pix / p.W_in, x = pix - y * p.W_in;
+            const int y = (int)(((uint32_t)pix * w_magic) >> 20), x = pix - y * p.W_in;
             const bool valid = env < p.n_env && y < p.H_out && x < p.W_out;
             __half* dst = p.out + ((size_t)env * p.P_out + (size_t)y * p.W_out + x) * 64;
+            env += d_env; pix += d_pix;
+            if (pix >= p.P_in) { pix -= p.P_in; ++env; }
             uint32_t v0[32], v1[32];
             const uint32_t taddr = tmem_d + grp * 64 + ((uint32_t)(q * 32) << 16);
             tmem_ld_32x32(taddr, v0);
@@ -147,12 +155,10 @@ conv_res_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                         for (int h = 0; h < 8; ++h) {
                             const int c = j + 2 * h;
-                            const float x0 = __uint_as_float(half ? v1[c] : v0[c]);
-                            const float x1 = __uint_as_float(half ? v1[c + 1] : v0[c + 1]);
-                            __half2 t = __floats2half2_rn(fmaf(x0, inv, s_bias[half * 32 + c]),
-                                                          fmaf(x1, inv, s_bias[half * 32 + c + 1]));
-                            t = __hmin2(__hmax2(t, __float2half2_rn(0.f)), __float2half2_rn(65504.f));
-                            pk[h] = *reinterpret_cast<uint32_t*>(&t);
+                            float x0 = __uint_as_float(half ? v1[c] : v0[c]);
+                            float x1 = __uint_as_float(half ? v1[c + 1] : v0[c + 1]);
+                            fma2(x0, x1, inv, s_bias[half * 32 + c], s_bias[half * 32 + c + 1]);
+                            pk[h] = relu_pack_h2(x0, x1);     // ReLU, round to fp16, clamp at the largest finite value
                         }
                         st_global_v8(dst + half * 32 + j, pk);
                     }
@@ -182,6 +188,7 @@ hts_status conv_res_launch(const CUtensorMap& act_map, const CUtensorMap& weight
     constexpr int NST = CPT == 2 ? 4 : 6;        // activation tiles in the ring: two being multiplied, the rest in flight
     const int smem = conv_res_smem_bytes(TAPS, CPT, p.tile_rows);
     if (smem > 227 * 1024) return HTS_ERR_SHAPE;
+    if (p.P_in < 1 || p.P_in > 2048 || p.W_in < 1 || p.W_in > 64) return HTS_ERR_SHAPE;   // the epilogue's row arithmetic
     if (smem > smem_set) {
         HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HTS_CUDA(cudaFuncSetAttribute(conv_res_kernel<TAPS, CPT, NST>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));

@@ -468,6 +468,8 @@ hts_status tc_check_geometry(const Geometry& g)
     if (rows2 > 256 || rows3 > 256) return HTS_ERR_SHAPE;                    // TMA box height
     if (conv_res_smem_bytes(4, 2, rows2) > 227 * 1024 || conv_res_smem_bytes(9, 1, rows3) > 227 * 1024) return HTS_ERR_SHAPE;
     if (g.F % BK) return HTS_ERR_SHAPE;
+    // row arithmetic of the conv2 / conv3 epilogues: grids of at most 2048 pixels, at most 64 wide
+    if (pl.P1s > 2048 || pl.W1s > 64 || g.H2 * g.W2 > 2048 || g.W2 > 64) return HTS_ERR_SHAPE;
     return HTS_OK;
 }
 

@@ -195,4 +195,24 @@ __host__ __device__ constexpr uint32_t instr_desc_f16(uint32_t ab_format, uint32
 }
 
 }  // namespace tc
+// fp32 pair -> packed fp16 pair with ReLU, saturating at the largest finite fp16
+__device__ __forceinline__ uint32_t relu_pack_h2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.relu.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// packed fp32 pairs (sm_100): two lanes of an add / fused multiply-add per instruction
+__device__ __forceinline__ void add2(float& a0, float& a1, float b0, float b1)
+{
+    asm("{\n\t.reg .b64 ra, rb;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
+        "add.rn.f32x2 ra, ra, rb;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fma2(float& a0, float& a1, float m, float c0, float c1)
+{
+    asm("{\n\t.reg .b64 ra, rm, rc;\n\tmov.b64 ra, {%0, %1};\n\tmov.b64 rm, {%2, %2};\n\tmov.b64 rc, {%3, %4};\n\t"
+        "fma.rn.f32x2 ra, ra, rm, rc;\n\tmov.b64 {%0, %1}, ra;\n\t}" : "+f"(a0), "+f"(a1) : "f"(m), "f"(c0), "f"(c1));
+}
+
 }  // namespace hts
