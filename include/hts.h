@@ -80,9 +80,9 @@ typedef struct {
  * packed-weight store and an activation workspace sized for max_batch (device
  * memory, freed by hts_policy_destroy).
  * A HTS_DTYPE_BF16 context (tensor-core kernels) takes C in {4, 8, 16} and frames
- * up to 260 pixels wide (the resident activation tiles of the second convolution
+ * up to 252 pixels wide (the resident activation tiles of the second convolution
  * must fit 227 KB of shared memory) whose first hidden layer, taken 2 x 2 pixels at a
- * time, has at most 2048 positions (260-wide frames up to 516 pixels high); anything else is refused here with
+ * time, has at most 2048 positions (252-wide frames up to 532 pixels high); anything else is refused here with
  * HTS_ERR_SHAPE, before any device call, never at step time.  Its frame buffers (obs, state_buffer) must start on a
  * 16-byte boundary (they are staged by TMA); a misaligned pointer is refused with
  * HTS_ERR_INVALID_ARG by the step calls.  Activations between layers are fp16: a

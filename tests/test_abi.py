@@ -52,8 +52,10 @@ def test_host_side_validation_needs_no_device():
     d = hts.hts_net_desc(4, 12, 12, 6, 1, 16)
     assert L.hts_policy_create(ctypes.byref(d), ctypes.byref(out)) == 2       # too small for the conv stack
     # shape limits of the tensor-core (bf16) kernels are checked at create time, before any device call
-    d = hts.hts_net_desc(4, 84, 264, 6, 1, 16)
+    d = hts.hts_net_desc(4, 84, 256, 6, 1, 16)
     assert L.hts_policy_create(ctypes.byref(d), ctypes.byref(out)) == 2       # wider than the resident conv2 tile allows
+    d = hts.hts_net_desc(4, 536, 252, 6, 1, 16)
+    assert L.hts_policy_create(ctypes.byref(d), ctypes.byref(out)) == 2       # first hidden grid over 2048 positions
     d = hts.hts_net_desc(3, 84, 84, 6, 1, 16)
     assert L.hts_policy_create(ctypes.byref(d), ctypes.byref(out)) == 2       # bf16 contexts take 4, 8 or 16 channels
     d = hts.hts_net_desc(12, 84, 84, 6, 1, 16)

@@ -114,7 +114,8 @@ def test_ragged_batch_sizes(n):
 @pytest.mark.parametrize("C,H,W,n", [(4, 64, 96, 77),     # 4 channels, width not 84: generic-width tensor-memory conv1; FC split 8
                                      (8, 84, 84, 33),     # 8 channels: shared-memory conv1 with two planes per tap
                                      (4, 36, 44, 150),    # image smaller than one 128-pixel tile: shared-memory conv1
-                                     (4, 100, 84, 41)])   # tiles straddle environments at other offsets (24 x 20 outputs)
+                                     (4, 100, 84, 41),    # tiles straddle environments at other offsets (24 x 20 outputs)
+                                     (4, 200, 252, 9)])   # widest frames: hidden grids of 25 x 31 and 23 x 30 positions
 def test_other_frame_shapes(C, H, W, n):
     import dataclasses
     cfg = dataclasses.replace(wl.CONFIGS[2], C=C, H=H, W=W)
