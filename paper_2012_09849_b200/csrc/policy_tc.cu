@@ -185,6 +185,150 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 
+// ---- FC for small batches with the weights resident: one CTA per (column tile, K range) and slot of row tiles.
+// A CTA asks for its whole weight slice (nk chunks of 128 x 64) before it waits for the previous kernel; a CTA of
+// this kernel cannot start before the previous kernel's CTA has left its SM, but the hand-over from the last of
+// those to the release of the wait (about 1.4 us) is enough for most of the slice.  After the wait only
+// activations cross the SM's L2 port: 112 KB per row tile instead of 224 KB.  Used while every CTA has one row
+// tile (n <= 640 for 4 x 84 x 84 frames: 31.0 against 31.5 us per step at n = 256, 51.2 against 52.7 us for 512
+// football frames); with two tiles per CTA it only equals the kernel above (one CTA per SM streams less from L2
+// than two do).  K ranges, the order inside them and the partial planes are those of the kernel above: the same
+// bits.
+constexpr int FCB_STAGES = 5;                   // activation chunks in flight (16 KiB each)
+constexpr int FCB_MAX_NK = 7;                   // weight chunks a CTA can keep: 7 x 16 KiB
+constexpr int FCB_MAX_TILES = 1;                // row tiles of a CTA (accumulators of 128 columns)
+constexpr int FCB_STAGE_FLOATS = 4 * 32 * 36;   // the epilogue warps' transposing buffers
+
+struct FcbParams {
+    int nk;                             // K chunks of one range
+    int n_env;                          // valid rows
+    int m_tiles;                        // row tiles of the batch
+    const float* inv_scale;
+    float* out_f32;                     // partial planes [range][rows][512]
+    size_t split_stride;
+    int* status;
+};
+
+__global__ void __launch_bounds__(192)
+fc_resident_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FcbParams p)
+{
+    constexpr int BN = 128;
+    constexpr int B_BYTES = BN * BK * 2;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t b_full[FCB_MAX_NK], a_full[FCB_STAGES], a_empty[FCB_STAGES], acc_full[FCB_MAX_TILES];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t* sm_a = sm + FCB_MAX_NK * B_BYTES;
+    const uint32_t a_base = base + FCB_MAX_NK * B_BYTES;
+    float* sm_stage = reinterpret_cast<float*>(sm_a + FCB_STAGES * A_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, range = blockIdx.y, slot = blockIdx.z, slots = gridDim.z;
+    const int my_tiles = slot < p.m_tiles ? (p.m_tiles - slot + slots - 1) / slots : 0;   // <= FCB_MAX_TILES (launcher)
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < FCB_MAX_NK; ++i) mbar_init(&b_full[i], 1);
+        for (int i = 0; i < FCB_STAGES; ++i) { mbar_init(&a_full[i], 1); mbar_init(&a_empty[i], 1); }
+        for (int i = 0; i < FCB_MAX_TILES; ++i) mbar_init(&acc_full[i], 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_slot, FCB_MAX_TILES * BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_slot;
+    if (warp == 0 && lane == 0) {                        // the weights do not depend on the previous kernel
+        for (int kc = 0; kc < p.nk; ++kc) {
+            mbar_arrive_expect_tx(&b_full[kc], B_BYTES);
+            tma_load_2d(sm + kc * B_BYTES, &tmB, (range * p.nk + kc) * BK, n0, &b_full[kc]);
+        }
+    }
+    pdl_wait();
+    pdl_trigger();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int t = 0; t < my_tiles; ++t) {
+                const int m0 = (slot + t * slots) * BM;
+                for (int kc = 0; kc < p.nk; ++kc, ++it) {
+                    const int s = it % FCB_STAGES;
+                    if (!mbar_wait(&a_empty[s], (((uint32_t)(it / FCB_STAGES)) & 1u) ^ 1u, abortp, p.status, 71)) { t = my_tiles; break; }
+                    mbar_arrive_expect_tx(&a_full[s], A_BYTES);
+                    tma_load_2d(sm_a + s * A_BYTES, &tmA, (range * p.nk + kc) * BK, m0, &a_full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_f16(0, BM, BN);
+            int it = 0;
+            bool alive = true;
+            for (int t = 0; alive && t < my_tiles; ++t) {
+                for (int kc = 0; kc < p.nk; ++kc, ++it) {
+                    const int s = it % FCB_STAGES;
+                    if (t == 0 && !mbar_wait(&b_full[kc], 0, abortp, p.status, 72)) { alive = false; break; }
+                    if (!mbar_wait(&a_full[s], ((uint32_t)(it / FCB_STAGES)) & 1u, abortp, p.status, 73)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(a_base + s * A_BYTES);
+                    const uint64_t bdesc = smem_desc_sw128(base + kc * B_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        mma_f16_ss(tmem_d + t * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (kc | k) != 0);
+                    mma_commit(&a_empty[s]);
+                }
+                if (alive) mma_commit(&acc_full[t]);
+            }
+        }
+    } else {
+        // epilogue warps 2..5: warp w may touch TMEM lanes [32*(w%4), 32*(w%4)+32)
+        const int q = warp & 3;
+        const float inv = *p.inv_scale;
+        float* stage = sm_stage + (warp - 2) * (32 * 36);
+        const int rl = lane >> 3, c4 = (lane & 7) * 4;
+        for (int t = 0; t < my_tiles; ++t) {
+            if (!mbar_wait_warp(&acc_full[t], 0, abortp, p.status, 74)) break;
+            tc_fence_after();
+            const int m0 = (slot + t * slots) * BM;
+            // one row per thread arrives; each warp turns its 32 x 32 blocks through shared memory so that eight
+            // lanes write one full 128-byte line
+            float* dst = p.out_f32 + range * p.split_stride + (size_t)(m0 + q * 32) * 512 + n0;
+#pragma unroll
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(tmem_d + ((uint32_t)(q * 32) << 16) + t * BN + c, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(stage + lane * 36 + j) =
+                        make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
+                                    __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + rl;
+                    const float4 val = *reinterpret_cast<const float4*>(stage + rr * 36 + c4);
+                    if (m0 + q * 32 + rr < p.n_env) *reinterpret_cast<float4*>(dst + (size_t)rr * 512 + c + c4) = val;
+                }
+                __syncwarp();
+            }
+        }
+    }
+    if (*abortp) {                                      // give copies still in flight time to land
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_d, FCB_MAX_TILES * BN);
+}
+
 // ---- FC for large batches: all K ranges of a tile in one CTA -----------------------------------------
 // The FC result is defined as  h = relu(bias + p_0 + p_1 + ... + p_{S-1}),  p_s = inv * (sum over the K chunks of
 // range s, accumulated in tensor memory in chunk order), the p_s added in index order in fp32.  Small batches
@@ -436,6 +580,22 @@ hts_status launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPar
     return HTS_OK;
 }
 
+hts_status launch_fc_resident(const CUtensorMap& a, const CUtensorMap& b, const FcbParams& p, int ranges, int slots,
+                              cudaStream_t s)
+{
+    constexpr int smem = FCB_MAX_NK * 128 * BK * 2 + FCB_STAGES * A_BYTES + FCB_STAGE_FLOATS * 4 + 1024;
+    static bool attr_set_by_device[kDeviceSlots] = {};
+    bool& attr_set = attr_set_by_device[device_slot()];
+    if (!attr_set) {
+        HTS_CUDA(cudaFuncSetAttribute(fc_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HTS_CUDA(cudaFuncSetAttribute(fc_resident_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+        attr_set = true;
+    }
+    HTS_CUDA(launch_pdl(fc_resident_kernel, dim3(4, ranges, slots), dim3(192), (size_t)smem, s, a, b, p));
+    note_launch();
+    return HTS_OK;
+}
+
 }  // namespace
 
 struct TcState {
@@ -593,7 +753,15 @@ hts_status tc_forward(TcState* t, const uint8_t* obs, const Indexing& ix, int n,
         HTS_CUDA(launch_pdl(fc_ranges_kernel, dim3(nblk(n, BM), 4), dim3(FCL_THREADS), (size_t)smem, s, t->mAfc, t->mBfc, fp));
         note_launch();
     } else {
-        st = launch_gemm<128, EPI_SPLITK>(t->mAfc, t->mBfc, p, dim3(nblk(n, BM), 4, t->splits), s);
+        // Weights resident per CTA when a K range is at most seven chunks and every CTA gets one row tile
+        const int m_tiles = (int)nblk(n, BM);
+        int slots = device_sm_count(device_slot()) / (4 * t->splits);
+        if (slots > m_tiles) slots = m_tiles;
+        if (t->cps <= FCB_MAX_NK && slots >= 1 && (m_tiles + slots - 1) / slots <= FCB_MAX_TILES) {
+            const FcbParams fp{t->cps, n, m_tiles, t->inv_scale + L_FC, t->hpart, (size_t)t->max_batch * 512, t->status};
+            st = launch_fc_resident(t->mAfc, t->mBfc, fp, t->splits, slots, s);
+        } else
+            st = launch_gemm<128, EPI_SPLITK>(t->mAfc, t->mBfc, p, dim3(nblk(n, BM), 4, t->splits), s);
         if (st != HTS_OK) return st;
     }
     prof.end(K_FC, s);
