@@ -80,6 +80,29 @@ def test_clipped_surrogate_gradient_both_sides_of_the_clip_range():
         pol.close()
 
 
+def test_full_size_batch_is_the_mean_of_its_halves():
+    """At the size bench.py times (1024 samples of the cfg3 network) the oracle's backward pass is out of reach; the
+    objective is a sample mean, so the gradient of a batch is the mean of the gradients of its halves, and a few
+    samples of the batch alone are checked against the oracle."""
+    cfg = dataclasses.replace(wl.CONFIGS[3], weight_dtype="fp32")
+    n = 1024
+    pol = Policy(cfg, max_batch=n)
+    try:
+        obs, actions, adv, ret = make_batch(cfg, n, 77)
+        whole = gpu_gradient(pol, obs, actions, adv, ret, None, 0.5, 0.01, 0.0)
+        h = n // 2
+        lo = gpu_gradient(pol, obs[:h], actions[:h], adv[:h], ret[:h], None, 0.5, 0.01, 0.0)
+        hi = gpu_gradient(pol, obs[h:], actions[h:], adv[h:], ret[h:], None, 0.5, 0.01, 0.0)
+        assert hts.hts_last_async_error(pol.ctx) == 0
+        for k in whole:
+            assert np.all(np.isfinite(whole[k])), k
+            assert rel_err(whole[k], 0.5 * (lo[k].astype(np.float64) + hi[k])) <= 1e-5, k
+        rows = np.array([0, 511, 512, 1023])
+        check(pol, obs[rows], actions[rows], adv[rows], ret[rows], None, 0.5, 0.01, 0.0)
+    finally:
+        pol.close()
+
+
 @pytest.mark.parametrize("C,H,W,A,n", [(8, 44, 52, 5, 7), (4, 84, 84, 18, 33), (16, 72, 96, 19, 4)])
 def test_other_shapes(C, H, W, A, n):
     cfg = dataclasses.replace(wl.CONFIGS[1], C=C, H=H, W=W, A=A)
